@@ -1,0 +1,196 @@
+/*
+ * mofq.h - C ABI of the B200 (sm_100a) MoFQ format-selection library.
+ *
+ * MoFQ = Mixture of Formats Quantization ("Integer or Floating Point? New Outlooks for Low-Bit
+ * Quantization on Large Language Models").  For every linear layer the library quantises the
+ * weight tensor (and, in the weight+activation setting, the calibration activations) onto the
+ * INT-k and FP-k grids of one bit-width with abs-max scales, reduces each candidate's error and
+ * keeps the candidate with the strictly smallest error (Algorithm 1).
+ *
+ * General conventions
+ *   - Every data pointer is a DEVICE pointer unless its comment says "host".  Structs that
+ *     describe tensors/layers/configs are read on the host.
+ *   - Tensors are row-major with leading dimension `ld` (elements).  Weights are [out, in]
+ *     (a Linear layer's weight, A_out = W * A_in, Section 3.2); activations are [tokens, in].
+ *   - `data` must be 16-byte aligned, `cols` a multiple of 8 and `ld` a multiple of 8.
+ *   - The caller owns every buffer, the workspace included; the library allocates nothing and
+ *     keeps no state between calls.  All work is enqueued on `stream` (a cudaStream_t passed as
+ *     void*; NULL = default stream) and the call returns without synchronising, unless stated.
+ *   - Return value: 0 on success, a negative MOFQ_ERR_* for a synchronous argument error (nothing
+ *     was enqueued).  Conditions found on the device (non-finite input, a reciprocal scale that
+ *     overflows binary32) are reported as MOFQ_STATUS_* bits in a device status word.
+ *   - Input values must be finite.
+ *
+ * Arithmetic contract (what "quantise" means here; the paper states round-to-nearest linear
+ * quantisation with abs-max scales and leaves the rest open):
+ *   absmax a of the scale block is exact; scale = RN32(a / Q), inv = RN32(Q / a) with
+ *   Q = 2^(k-1)-1 (INT) or the largest finite magnitude of the FP grid; an all-zero block has
+ *   scale = inv = 1.  t = RN32(x * inv).  INT code = RNE(t) as k-bit two's complement.  FP code =
+ *   nearest grid magnitude to |t| (ties to the even code), sign bit copied from x.  With
+ *   caller-supplied scales inv = RN32(1 / scale) and out-of-range values saturate.  The error of
+ *   a candidate is mean (x - value(code) * scale)^2 over the whole tensor.
+ */
+#ifndef MOFQ_H
+#define MOFQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOFQ_MAX_CAND 4 /* most candidate formats per call */
+
+/* Number formats (Section 2; Section 4.2 and Table 3 for the two FP4 variants). */
+typedef enum {
+    MOFQ_INT4 = 0,          /* two's complement, codes -8..7, abs-max maps to 7                     */
+    MOFQ_INT8 = 1,          /* two's complement, codes -128..127, abs-max maps to 127               */
+    MOFQ_FP4_E2M1 = 2,      /* Table 3 "w/o NaN&Inf": 0 .5 1 1.5 2 3 4 6 and negatives, max 6       */
+    MOFQ_FP4_E2M1_IEEE = 3, /* Table 3 "w/ NaN&Inf": exponent field 3 reserved, max 3               */
+    MOFQ_FP8_E4M3 = 4,      /* bias 7, only S.1111.111 reserved, max 448 (hardware-compatible)      */
+    MOFQ_FP8_E5M2 = 5       /* bias 15, exponent field 31 reserved, max 57344                       */
+} mofq_format;
+
+/* Scale granularity (Section 3.2: per-channel weights, per-tensor activations; per-group =
+ * `group` consecutive elements along the input dimension, cols % group == 0, group % 8 == 0). */
+typedef enum { MOFQ_PER_TENSOR = 0, MOFQ_PER_CHANNEL = 1, MOFQ_PER_GROUP = 2 } mofq_gran;
+#define MOFQ_GRAN_NONE (-1)
+
+typedef enum { MOFQ_F16 = 0, MOFQ_BF16 = 1 } mofq_dtype;
+
+/* Error metric of Algorithm 1 (Section 4.1: tensor error or layer output error). */
+typedef enum { MOFQ_TENSOR_MSE = 0, MOFQ_LAYER_OUTPUT_MSE = 1 } mofq_metric;
+
+/* Synchronous error codes. */
+#define MOFQ_OK 0
+#define MOFQ_ERR_INVALID_ARG (-1)         /* NULL pointer, non-positive size, bad enum, too many candidates  */
+#define MOFQ_ERR_UNSUPPORTED (-2)         /* candidate bit-width != bit_width, cols % group != 0, ...         */
+#define MOFQ_ERR_MISALIGNED (-3)          /* data not 16-byte aligned, or cols / ld not a multiple of 8       */
+#define MOFQ_ERR_WORKSPACE_TOO_SMALL (-4) /* workspace_bytes below the matching *_workspace_bytes() value     */
+#define MOFQ_ERR_CUDA (-5)                /* a CUDA runtime call or kernel launch failed                      */
+
+/* Asynchronous status bits (device status word / mofq_result.status). */
+#define MOFQ_STATUS_NONFINITE_INPUT 1 /* an Inf or NaN was found in the input           */
+#define MOFQ_STATUS_SCALE_OVERFLOW 2  /* Q / absmax is not finite in binary32           */
+#define MOFQ_STATUS_TIMEOUT 4         /* a bounded device-side wait expired             */
+
+typedef struct {
+    const void *data; /* device, row-major                           */
+    int32_t dtype;    /* mofq_dtype                                  */
+    int32_t reserved;
+    int64_t rows, cols, ld;
+} mofq_tensor;
+
+/* One linear layer: W [out, in]; X [tokens, in] calibration activations (data == NULL when the
+ * metric does not need them). */
+typedef struct {
+    mofq_tensor W;
+    mofq_tensor X;
+} mofq_layer;
+
+/* The arguments of Algorithm 1: MoFQ(model, is_w_only, format_candidates, bit_width, error_metric)
+ * plus the scale granularities. */
+typedef struct {
+    int32_t bit_width;                 /* 4 or 8; every candidate must have this width                 */
+    int32_t n_candidates;              /* 1..MOFQ_MAX_CAND                                              */
+    int32_t candidates[MOFQ_MAX_CAND]; /* mofq_format, in the caller's order: ties go to the first      */
+    int32_t is_w_only;                 /* 1: quantise W only; 0: W and X (same format for both)         */
+    int32_t w_gran;                    /* mofq_gran for W                                               */
+    int32_t w_group;                   /* group size when a W granularity is MOFQ_PER_GROUP             */
+    int32_t w_gran2;                   /* MOFQ_GRAN_NONE, or a second W granularity scored from the     */
+                                       /* same read (tensor metric only); results then hold 2 records   */
+                                       /* per layer: [layer][0] for w_gran, [layer][1] for w_gran2      */
+    int32_t a_gran;                    /* mofq_gran for X (MOFQ_PER_TENSOR in the paper)                */
+    int32_t a_group;
+    int32_t metric;                    /* mofq_metric                                                   */
+} mofq_config;
+
+/* One selection record (device memory). */
+typedef struct {
+    int32_t chosen;             /* index into mofq_config.candidates                                    */
+    int32_t status;             /* MOFQ_STATUS_* bits                                                   */
+    float error[MOFQ_MAX_CAND]; /* MSE per candidate, caller's order                                    */
+    float nsr[MOFQ_MAX_CAND];   /* layer metric only: sum (Y-Yq)^2 / sum Y^2 (noise/signal power)       */
+    float rel_margin;           /* (second smallest - smallest) / smallest; +Inf if smallest is 0       */
+    int32_t reserved;
+} mofq_result;
+
+/*
+ * mofq_quantize_tensor - round-to-nearest linear quantisation of one tensor to one format
+ * (Section 1 "naive linear quantization with round-to-nearest", Algorithm 1 `quantize_layer`;
+ * granularities Section 3.2).
+ *   x           tensor to quantise
+ *   scales_in   NULL: abs-max scales are derived.  Else device array of n_scales floats
+ *               (calibration scales, Section 3.2 dynamic tensor analysis); values saturate.
+ *   codes_out   nullable.  8-bit formats: rows*cols bytes.  4-bit: rows*cols/2 bytes, element 2j in
+ *               the low nibble of byte j.  Dense (leading dimension = cols).  INT codes are two's
+ *               complement; FP codes are sign|exponent|mantissa with Table 3's numbering.
+ *   scales_out  nullable.  n_scales floats: [1], [rows] or [rows, cols/group] row-major.
+ *   dequant_out nullable.  rows*cols elements of x's dtype: RN32(value*scale) rounded to nearest even.
+ *   workspace   at least mofq_tensor_workspace_bytes(x) bytes, 256-byte aligned.  On completion
+ *               the first int32 of the workspace holds the MOFQ_STATUS_* bits of this call.
+ */
+int mofq_quantize_tensor(const mofq_tensor *x, int format, int gran, int group, const float *scales_in,
+                         void *codes_out, float *scales_out, void *dequant_out,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * mofq_tensor_error - tensor MSE of n candidate formats of one bit-width from ONE read of x
+ * (Section 3.2 static tensor analysis: "mean squared error between quantized and original
+ * tensors"; Algorithm 1 `compute_error` with the tensor metric).
+ *   formats     host array of n mofq_format values of equal bit-width
+ *   gran2       MOFQ_GRAN_NONE or a second granularity scored from the same read
+ *   mse_out     device, n floats (2n when gran2 is given: [gran][candidate])
+ *   workspace   at least mofq_tensor_workspace_bytes(x); first int32 = status bits on completion
+ */
+int mofq_tensor_error(const mofq_tensor *x, const int32_t *formats, int n, int gran, int gran2, int group,
+                      float *mse_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * mofq_layer_output_error - error of the layer output Y = X W^T when its inputs are quantised
+ * (Section 3.2 layer analysis; Algorithm 1 `compute_error` with the layer output metric).
+ * is_w_only: Yq = X dq(W)^T; otherwise Yq = dq(X) dq(W)^T with the same format for both tensors.
+ *   mse_out, nsr_out   device, cfg->n_candidates floats each, caller's order
+ *   workspace          at least mofq_workspace_bytes(L, 1, cfg); first int32 = status bits
+ */
+int mofq_layer_output_error(const mofq_layer *L, const mofq_config *cfg, float *mse_out, float *nsr_out,
+                            void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * mofq_select_formats - Algorithm 1 over a model's layer list: score every candidate on every
+ * layer and keep the strict minimum in the caller's candidate order.
+ *   layers       host array of n_layers descriptors (device tensors)
+ *   results_out  device array of n_layers records (2*n_layers when cfg->w_gran2 is given)
+ *   workspace    at least mofq_workspace_bytes(layers, n_layers, cfg)
+ */
+int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_config *cfg,
+                        mofq_result *results_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * mofq_select_formats_host - the same selection for a model whose tensors live in HOST memory
+ * (pinned memory recommended).  Layer data pointers are host pointers and the tensors are dense
+ * (ld == cols); the call copies each layer into a staging area of the device workspace, scores it
+ * there, copies the records back and SYNCHRONISES before returning.
+ *   results_host host array of n_layers (or 2*n_layers) records
+ *   workspace    device, at least mofq_host_workspace_bytes(layers, n_layers, cfg)
+ */
+int mofq_select_formats_host(const mofq_layer *layers_host_data, int n_layers, const mofq_config *cfg,
+                             mofq_result *results_host, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Workspace sizes in bytes (host-side arithmetic only). */
+size_t mofq_tensor_workspace_bytes(const mofq_tensor *x);
+size_t mofq_workspace_bytes(const mofq_layer *layers, int n_layers, const mofq_config *cfg);
+size_t mofq_host_workspace_bytes(const mofq_layer *layers, int n_layers, const mofq_config *cfg);
+
+/* Static facts about a format: bit-width (4/8) and largest finite magnitude; -1 / 0 for a bad enum. */
+int mofq_format_bits(int format);
+float mofq_format_max(int format);
+
+/* Human-readable name of a MOFQ_ERR_* code. */
+const char *mofq_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOFQ_H */

@@ -1,0 +1,82 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "mofq.h"
+
+namespace mofq {
+
+// ---- format description used by the kernels ------------------------------------------------------
+// FP grid with E exponent bits, M mantissa bits, bias 2^(E-1)-1 (Section 2; Table 3 for E2M1):
+//   Q      largest finite magnitude (abs-max maps here)
+//   eminb  binary32 exponent field of the smallest normal 2^(1-bias), shifted into place
+//   kadd   (23 - M) << 23: added to an exponent field it yields the power of two whose ulp is the
+//          grid spacing of that binade
+struct FmtDesc {
+    int is_fp, bits, M, bias;
+    float Q;
+    uint32_t eminb, kadd;
+    float min_normal;
+};
+
+// Candidate set in canonical slot order: [INT (if any)] [FP 0] [FP 1].
+struct CandSet {
+    int n_int, n_fp;
+    float int_q;
+    float fp_q[2];
+    uint32_t fp_eminb[2], fp_kadd[2];
+};
+
+constexpr int kMaxAcc = 8;        // accumulators per block: up to 2 granularities x 3 canonical slots (padded)
+constexpr int kMaxSlots = 2048;   // most thread blocks a scoring kernel is launched with
+
+// Header of the scoring workspace (device).  Zero before the first launch; every kernel that uses
+// it leaves counter and absmax_bits zero again, and the last block moves `status` into the output.
+struct WsHeader {
+    int32_t status;        // MOFQ_STATUS_* bits of the running call
+    uint32_t counter;      // blocks finished (last-block-done reduction)
+    uint32_t absmax_bits;  // per-tensor abs-max as a 16-bit magnitude pattern
+    uint32_t pad[61];
+};
+static_assert(sizeof(WsHeader) == 256, "header is one 256-byte line");
+
+// What the last block writes once all partial sums are in.
+struct Finalize {
+    float *mse_out;        // nullable: [set][candidate] floats, caller's order
+    mofq_result *res;      // nullable: one record per set
+    int32_t *status_out;   // nullable: receives the status bits (else they stay in the header)
+    int n_cand, n_sets, nc;
+    int perm[MOFQ_MAX_CAND];   // caller's candidate index -> canonical slot
+    double inv_n;          // 1 / element count
+};
+
+struct ScoreJob {
+    mofq_tensor x;
+    CandSet cs;
+    int gran, gran2, group;    // gran2 = MOFQ_GRAN_NONE or second granularity
+    Finalize fin;
+    WsHeader *hdr;
+    double *partials;          // kMaxSlots * kMaxAcc doubles
+};
+
+inline size_t score_ws_bytes() { return sizeof(WsHeader) + sizeof(double) * kMaxSlots * kMaxAcc; }
+
+bool describe_format(int format, FmtDesc *d);
+int build_candset(const int32_t *formats, int n, int bit_width, CandSet *cs, int *perm, int *nc);
+int sm_count();
+
+// kernels' host launchers (mofq_kq.cu)
+int launch_score(const ScoreJob &job, cudaStream_t st);
+int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in,
+                void *codes_out, float *scales_out, void *dequant_out, void *values_out, int values_dtype,
+                WsHeader *hdr, cudaStream_t st);
+
+// layer-output metric (mofq_layer.cu): extra workspace beyond the scoring workspace, and one layer's run.
+// Exactly one of `res` (selection record) or `mse_out`/`nsr_out` (raw errors, caller's order) is given.
+size_t layer_metric_ws_bytes(const mofq_layer *layers, int n_layers, const mofq_config *cfg);
+int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *res, float *mse_out, float *nsr_out,
+                     void *workspace, size_t workspace_bytes, cudaStream_t st);
+
+}  // namespace mofq

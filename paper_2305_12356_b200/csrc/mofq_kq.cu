@@ -1,0 +1,732 @@
+// Quantise / score kernels: abs-max scale -> round to the INT-k and FP-k grids -> dequantise ->
+// squared error -> block reduce, for all candidates from one read of the tensor.
+//
+// The arithmetic follows the contract in mofq.h: scale = RN32(a/Q), inv = RN32(Q/a),
+// t = RN32(x*inv), INT: RNE(t); FP: RNE of |t| onto the spacing 2^(e-M) of its binade, e clamped
+// at the smallest normal exponent (gradual underflow).  Both roundings use the add-and-subtract
+// of a power of two whose ulp equals the wanted spacing, which is an exact RNE in binary32.
+// Because every grid is symmetric, (x - v*s)^2 = (|x| - |v|*s)^2 and the scoring kernels work on
+// magnitudes only; signs matter only when codes are written out.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <algorithm>
+#include <type_traits>
+
+#include "mofq_internal.h"
+
+namespace mofq {
+namespace {
+
+constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds |t| < 2^22 to an integer (RNE)
+
+// ---- small device helpers --------------------------------------------------------------------------
+template <int DT>
+__device__ __forceinline__ void unpack2(uint32_t w, float &lo, float &hi)
+{
+    if (DT == MOFQ_F16) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w));
+        lo = f.x;
+        hi = f.y;
+    } else {
+        lo = __uint_as_float(w << 16);
+        hi = __uint_as_float(w & 0xFFFF0000u);
+    }
+}
+
+// 16-bit magnitude pattern -> float (exact)
+template <int DT>
+__device__ __forceinline__ float mag16_to_float(uint32_t m16)
+{
+    if (DT == MOFQ_F16) return __half2float(__ushort_as_half((unsigned short)m16));
+    return __uint_as_float(m16 << 16);
+}
+
+template <int DT>
+__device__ __forceinline__ bool mag16_nonfinite(uint32_t m16)
+{
+    return m16 >= (DT == MOFQ_F16 ? 0x7C00u : 0x7F80u);
+}
+
+// running abs-max over packed 16-bit magnitude patterns (integer order == magnitude order; Inf/NaN sort on top)
+__device__ __forceinline__ uint32_t absmax_chunk(const uint4 v, uint32_t m)
+{
+    m = __vmaxu2(m, v.x & 0x7FFF7FFFu);
+    m = __vmaxu2(m, v.y & 0x7FFF7FFFu);
+    m = __vmaxu2(m, v.z & 0x7FFF7FFFu);
+    m = __vmaxu2(m, v.w & 0x7FFF7FFFu);
+    return m;
+}
+__device__ __forceinline__ uint32_t fold16(uint32_t m) { return max(m & 0xFFFFu, m >> 16); }
+
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem)
+{
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+}
+
+template <int NC>
+struct Scales {
+    float s[NC], inv[NC];
+};
+
+__device__ __forceinline__ void scale_pair(float a, float Q, float &s, float &inv, int &status)
+{
+    if (a == 0.0f) {
+        s = 1.0f;
+        inv = 1.0f;
+    } else {
+        s = __fdiv_rn(a, Q);
+        inv = __fdiv_rn(Q, a);
+        if (isinf(inv)) status |= MOFQ_STATUS_SCALE_OVERFLOW;
+    }
+}
+
+template <int NI, int NFP>
+__device__ __forceinline__ void make_scales(float a, const CandSet &c, Scales<NI + NFP> &sc, int &status)
+{
+    if (NI) scale_pair(a, c.int_q, sc.s[0], sc.inv[0], status);
+#pragma unroll
+    for (int f = 0; f < NFP; ++f) scale_pair(a, c.fp_q[f], sc.s[NI + f], sc.inv[NI + f], status);
+}
+
+// |t| -> nearest FP grid magnitude (RNE), no saturation (|t| <= Q(1+2^-23) under abs-max scales)
+__device__ __forceinline__ float fp_grid_round(float t, uint32_t eminb, uint32_t kadd)
+{
+    const uint32_t eb = max(__float_as_uint(t) & 0x7F800000u, eminb);
+    const float c = __uint_as_float(eb + kadd);
+    return __fsub_rn(__fadd_rn(t, c), c);
+}
+
+// one magnitude a = |x| scored against every candidate
+template <int NI, int NFP>
+__device__ __forceinline__ void score1(float a, const Scales<NI + NFP> &sc, const CandSet &c, float *acc)
+{
+    if (NI) {
+        const float t = __fmul_rn(a, sc.inv[0]);
+        const float r = __fsub_rn(__fadd_rn(t, kMagic), kMagic);
+        const float e = __fmaf_rn(-r, sc.s[0], a);
+        acc[0] = __fmaf_rn(e, e, acc[0]);
+    }
+#pragma unroll
+    for (int f = 0; f < NFP; ++f) {
+        const float t = __fmul_rn(a, sc.inv[NI + f]);
+        const float r = fp_grid_round(t, c.fp_eminb[f], c.fp_kadd[f]);
+        const float e = __fmaf_rn(-r, sc.s[NI + f], a);
+        acc[NI + f] = __fmaf_rn(e, e, acc[NI + f]);
+    }
+}
+
+template <int DT, int NI, int NFP>
+__device__ __forceinline__ void score_chunk(const uint4 v, const Scales<NI + NFP> &sc, const CandSet &c, float *acc)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float lo, hi;
+        unpack2<DT>(w[i], lo, hi);
+        score1<NI, NFP>(fabsf(lo), sc, c, acc);
+        score1<NI, NFP>(fabsf(hi), sc, c, acc);
+    }
+}
+
+// ---- block reductions and the last-block-done finish -------------------------------------------------
+__device__ __forceinline__ uint32_t block_max_u32(uint32_t v, uint32_t *red /* >= 33 words */)
+{
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t r = lane < nw ? red[lane] : 0u;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) r = max(r, __shfl_xor_sync(0xffffffffu, r, o));
+        if (lane == 0) red[32] = r;
+    }
+    __syncthreads();
+    return red[32];
+}
+
+// Sum NA doubles per thread over the block in a fixed order; the totals land in red[0..NA).
+template <int NA>
+__device__ __forceinline__ void block_sum(double *acc, double *red /* >= 32*NA + NA doubles */)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int j = 0; j < NA; ++j)
+#pragma unroll
+        for (int o = 16; o; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+    __syncthreads();
+    if (lane == 0)
+        for (int j = 0; j < NA; ++j) red[NA + warp * NA + j] = acc[j];
+    __syncthreads();
+    if (threadIdx.x < NA) {
+        double s = 0.0;
+        for (int w = 0; w < nw; ++w) s += red[NA + w * NA + threadIdx.x];
+        red[threadIdx.x] = s;
+    }
+    __syncthreads();
+}
+
+__device__ void write_outputs(const double *tot, const Finalize &fin, WsHeader *hdr)
+{
+    int status = 0;
+    if (fin.res) status = atomicExch(&hdr->status, 0);
+    for (int s = 0; s < fin.n_sets; ++s) {
+        double err[MOFQ_MAX_CAND];
+        for (int i = 0; i < fin.n_cand; ++i) {
+            err[i] = tot[s * fin.nc + fin.perm[i]] * fin.inv_n;
+            if (fin.mse_out) fin.mse_out[s * fin.n_cand + i] = (float)err[i];
+        }
+        if (fin.res) {
+            // Algorithm 1: min_error = inf; replace only on a strictly smaller error, caller's order
+            double best = INFINITY, second = INFINITY;
+            int chosen = -1;
+            for (int i = 0; i < fin.n_cand; ++i) {
+                if (err[i] < best) {
+                    second = best;
+                    best = err[i];
+                    chosen = i;
+                } else if (err[i] < second) {
+                    second = err[i];
+                }
+            }
+            mofq_result r;
+            r.chosen = chosen;
+            r.status = status;
+            for (int i = 0; i < MOFQ_MAX_CAND; ++i) {
+                r.error[i] = i < fin.n_cand ? (float)err[i] : 0.0f;
+                r.nsr[i] = 0.0f;
+            }
+            r.rel_margin = best > 0.0 ? (float)((second - best) / best) : INFINITY;
+            r.reserved = 0;
+            fin.res[s] = r;
+        }
+    }
+}
+
+// Every block deposits its partial sums; the block that arrives last adds them in slot order.
+template <int NA>
+__device__ void block_finish(double *acc, int status, WsHeader *hdr, double *partials, const Finalize &fin, double *red)
+{
+    __shared__ int is_last;
+    if (status) atomicOr(&hdr->status, status);
+    block_sum<NA>(acc, red);
+    if (threadIdx.x == 0) {
+        for (int j = 0; j < NA; ++j) partials[(size_t)blockIdx.x * kMaxAcc + j] = red[j];
+        __threadfence();
+        const uint32_t ticket = atomicAdd(&hdr->counter, 1u);
+        is_last = (ticket == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double tot[NA];
+#pragma unroll
+    for (int j = 0; j < NA; ++j) tot[j] = 0.0;
+    for (int slot = threadIdx.x; slot < (int)gridDim.x; slot += blockDim.x)
+#pragma unroll
+        for (int j = 0; j < NA; ++j) tot[j] += __ldcg(&partials[(size_t)slot * kMaxAcc + j]);
+    block_sum<NA>(tot, red);
+    if (threadIdx.x == 0) {
+        hdr->counter = 0;
+        write_outputs(red, fin, hdr);
+    }
+}
+
+// ---- scoring kernel 1: dense tensor, per-group scales -------------------------------------------------
+// A tile is 128 consecutive groups staged in shared memory; thread g owns group g and walks its
+// 16-byte chunks in an order rotated by g, which keeps the quarter-warps on distinct banks.
+constexpr int kGroupsPerTile = 128;
+
+template <int DT, int NI, int NFP>
+__global__ void __launch_bounds__(kGroupsPerTile)
+kq_score_groups(const uint16_t *__restrict__ x, long long n_groups, int group, CandSet cs, WsHeader *hdr,
+                double *partials, Finalize fin)
+{
+    constexpr int NC = NI + NFP;
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ double red[33 * NC];
+    const int cpg = group >> 3;  // 16-byte chunks per group (power of two)
+    const long long n_tiles = (n_groups + kGroupsPerTile - 1) / kGroupsPerTile;
+    double dacc[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) dacc[j] = 0.0;
+    int status = 0;
+
+    for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const long long g0 = tile * kGroupsPerTile;
+        const int ng = (int)min((long long)kGroupsPerTile, n_groups - g0);
+        const int chunks = ng * cpg;
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(x) + (size_t)g0 * group * 2;
+        for (int q = threadIdx.x; q < chunks; q += kGroupsPerTile) cp_async16(smem + q * 16, src + (size_t)q * 16);
+        cp_async_wait_all();
+        __syncthreads();
+        if ((int)threadIdx.x < ng) {
+            const uint4 *base = reinterpret_cast<const uint4 *>(smem) + threadIdx.x * cpg;
+            uint32_t m = 0;
+            for (int j = 0; j < cpg; ++j) m = absmax_chunk(base[(j + threadIdx.x) & (cpg - 1)], m);
+            const uint32_t m16 = fold16(m);
+            if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+            Scales<NC> sc;
+            make_scales<NI, NFP>(mag16_to_float<DT>(m16), cs, sc, status);
+            float acc[NC];
+#pragma unroll
+            for (int j = 0; j < NC; ++j) acc[j] = 0.0f;
+            for (int j = 0; j < cpg; ++j) score_chunk<DT, NI, NFP>(base[(j + threadIdx.x) & (cpg - 1)], sc, cs, acc);
+#pragma unroll
+            for (int j = 0; j < NC; ++j) dacc[j] += (double)acc[j];
+        }
+        __syncthreads();
+    }
+    block_finish<NC>(dacc, status, hdr, partials, fin, red);
+}
+
+// ---- scoring kernel 2: one row per block; per-channel and/or per-group scales ---------------------------
+// The row is staged in shared memory so that the abs-max pass and the scoring pass cost one HBM read.
+// Accumulator order: [first set][second set]; `grp_first` says whether the group set comes first.
+constexpr int kRowThreads = 256;
+
+template <int DT, int NI, int NFP, bool CH, bool GRP>
+__global__ void __launch_bounds__(kRowThreads)
+kq_score_rows(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, int group, int grp_first,
+              CandSet cs, WsHeader *hdr, double *partials, Finalize fin)
+{
+    constexpr int NC = NI + NFP;
+    constexpr int NA = NC * ((CH ? 1 : 0) + (GRP ? 1 : 0));
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ double red[33 * NA];
+    __shared__ uint32_t mred[34];
+    __shared__ Scales<NC> row_sc;
+    __shared__ int row_status;
+    const int chunks = cols >> 3;
+    const int cpg = GRP ? (group >> 3) : 1;
+    const int gpr = GRP ? cols / group : 0;
+    uint16_t *gmax = reinterpret_cast<uint16_t *>(smem + (size_t)cols * 2);  // per-group abs-max patterns
+    const uint4 *row4 = reinterpret_cast<const uint4 *>(smem);
+    double dacc[NA];
+#pragma unroll
+    for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
+    int status = 0;
+
+    for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(x + row * ld);
+        for (int q = threadIdx.x; q < chunks; q += kRowThreads) cp_async16(smem + q * 16, src + (size_t)q * 16);
+        cp_async_wait_all();
+        __syncthreads();
+        // pass 1: abs-max
+        uint32_t m16 = 0;
+        if (GRP) {
+            for (int g = threadIdx.x; g < gpr; g += kRowThreads) {
+                const uint4 *base = row4 + g * cpg;
+                uint32_t m = 0;
+                for (int j = 0; j < cpg; ++j) m = absmax_chunk(base[(j + g) & (cpg - 1)], m);
+                const uint32_t gm = fold16(m);
+                gmax[g] = (uint16_t)gm;
+                m16 = max(m16, gm);
+            }
+        } else {
+            uint32_t m = 0;
+            for (int q = threadIdx.x; q < chunks; q += kRowThreads) m = absmax_chunk(row4[q], m);
+            m16 = fold16(m);
+        }
+        if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+        if (CH) {
+            const uint32_t rm = block_max_u32(m16, mred);
+            if (threadIdx.x == 0) {
+                int st = 0;
+                make_scales<NI, NFP>(mag16_to_float<DT>(rm), cs, row_sc, st);
+                row_status = st;
+            }
+            __syncthreads();
+            status |= row_status;
+        }
+        // pass 2: score
+        float acc_g[NC], acc_c[NC];  // group-scale and channel-scale candidates
+#pragma unroll
+        for (int j = 0; j < NC; ++j) acc_g[j] = acc_c[j] = 0.0f;
+        if (GRP) {
+            Scales<NC> rsc;
+            if (CH) rsc = row_sc;
+            for (int g = threadIdx.x; g < gpr; g += kRowThreads) {
+                const uint4 *base = row4 + g * cpg;
+                Scales<NC> gsc;
+                make_scales<NI, NFP>(mag16_to_float<DT>(gmax[g]), cs, gsc, status);
+                for (int j = 0; j < cpg; ++j) {
+                    const uint4 v = base[(j + g) & (cpg - 1)];
+                    score_chunk<DT, NI, NFP>(v, gsc, cs, acc_g);
+                    if (CH) score_chunk<DT, NI, NFP>(v, rsc, cs, acc_c);
+                }
+            }
+        } else {
+            const Scales<NC> rsc = row_sc;
+            for (int q = threadIdx.x; q < chunks; q += kRowThreads) score_chunk<DT, NI, NFP>(row4[q], rsc, cs, acc_c);
+        }
+        if (CH && GRP) {
+#pragma unroll
+            for (int j = 0; j < NC; ++j) {
+                dacc[j] += (double)(grp_first ? acc_g[j] : acc_c[j]);
+                dacc[NC + j] += (double)(grp_first ? acc_c[j] : acc_g[j]);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < NC; ++j) dacc[j] += (double)(GRP ? acc_g[j] : acc_c[j]);
+        }
+        __syncthreads();
+    }
+    block_finish<NA>(dacc, status, hdr, partials, fin, red);
+}
+
+// ---- per-tensor scale: abs-max kernel, then a streaming scoring kernel -----------------------------------
+template <int DT>
+__global__ void __launch_bounds__(256)
+kq_absmax(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, WsHeader *hdr)
+{
+    uint32_t m = 0;
+    const long long total = rows * chunks_per_row;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / chunks_per_row;
+        const int c = (int)(i - r * chunks_per_row);
+        m = absmax_chunk(__ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c), m);
+    }
+    uint32_t m16 = fold16(m);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) m16 = max(m16, __shfl_xor_sync(0xffffffffu, m16, o));
+    if ((threadIdx.x & 31) == 0 && m16) atomicMax(&hdr->absmax_bits, m16);
+}
+
+template <int DT, int NI, int NFP>
+__global__ void __launch_bounds__(256)
+kq_score_uniform(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, CandSet cs,
+                 WsHeader *hdr, double *partials, Finalize fin)
+{
+    constexpr int NC = NI + NFP;
+    __shared__ double red[33 * NC];
+    int status = 0;
+    const uint32_t m16 = *reinterpret_cast<volatile uint32_t *>(&hdr->absmax_bits);
+    if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+    Scales<NC> sc;
+    make_scales<NI, NFP>(mag16_to_float<DT>(m16), cs, sc, status);
+    double dacc[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) dacc[j] = 0.0;
+    const long long total = rows * chunks_per_row;
+    int n = 0;
+    float acc[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) acc[j] = 0.0f;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / chunks_per_row;
+        const int c = (int)(i - r * chunks_per_row);
+        score_chunk<DT, NI, NFP>(__ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c), sc, cs, acc);
+        if (++n == 16) {  // keep the binary32 chains short: 128 terms, then fold into double
+#pragma unroll
+            for (int j = 0; j < NC; ++j) {
+                dacc[j] += (double)acc[j];
+                acc[j] = 0.0f;
+            }
+            n = 0;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < NC; ++j) dacc[j] += (double)acc[j];
+    block_finish<NC>(dacc, status, hdr, partials, fin, red);
+}
+
+// ---- emit kernel: codes / scales / dequantised values for ONE format ---------------------------------------
+// One row per block.  GRAN selects where the scale of a 16-byte chunk comes from.
+__device__ __forceinline__ uint32_t fp_code_from_mag(float r, const FmtDesc &f)
+{
+    // below the smallest normal, adding it puts the subnormal step count into the mantissa field
+    uint32_t rb = (r < f.min_normal) ? __float_as_uint(__fadd_rn(r, f.min_normal)) - (1u << 23) : __float_as_uint(r);
+    return (rb >> (23 - f.M)) - ((uint32_t)(127 - f.bias) << f.M);
+}
+
+template <int DT>
+__device__ __forceinline__ uint16_t to_storage(float v)
+{
+    if (DT == MOFQ_F16) return __half_as_ushort(__float2half_rn(v));
+    return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+
+template <int DT, int GRAN>
+__global__ void __launch_bounds__(kRowThreads)
+kq_emit(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, FmtDesc f, int group,
+        const float *__restrict__ scales_in, unsigned char *codes_out, float *scales_out, uint16_t *dequant_out,
+        uint16_t *values_out, int values_dtype, WsHeader *hdr)
+{
+    __shared__ uint32_t mred[34];
+    const int chunks = cols >> 3;
+    const int lanes_per_group = GRAN == MOFQ_PER_GROUP ? (group >> 3) : 1;  // power of two <= 32
+    const int gpr = GRAN == MOFQ_PER_GROUP ? cols / group : 1;
+    int status = 0;
+    const float int_lo = -f.Q - 1.0f;
+
+    for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
+        const uint4 *xr = reinterpret_cast<const uint4 *>(x + row * ld);
+        float s = 1.0f, inv = 1.0f;
+        if (GRAN == MOFQ_PER_TENSOR || GRAN == MOFQ_PER_CHANNEL) {
+            if (scales_in) {
+                s = scales_in[GRAN == MOFQ_PER_TENSOR ? 0 : row];
+                inv = __fdiv_rn(1.0f, s);
+            } else {
+                uint32_t m16;
+                if (GRAN == MOFQ_PER_TENSOR) {
+                    m16 = *reinterpret_cast<volatile uint32_t *>(&hdr->absmax_bits);
+                } else {
+                    uint32_t m = 0;
+                    for (int q = threadIdx.x; q < chunks; q += kRowThreads) m = absmax_chunk(__ldg(xr + q), m);
+                    m16 = block_max_u32(fold16(m), mred);
+                }
+                if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+                scale_pair(mag16_to_float<DT>(m16), f.Q, s, inv, status);
+            }
+            if (scales_out && threadIdx.x == 0 && (GRAN == MOFQ_PER_CHANNEL || row == 0))
+                scales_out[GRAN == MOFQ_PER_TENSOR ? 0 : row] = s;
+        }
+        const int iters = (chunks + kRowThreads - 1) / kRowThreads;
+        for (int it = 0; it < iters; ++it) {
+            const int q = it * kRowThreads + threadIdx.x;
+            const bool active = q < chunks;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (active) v = __ldg(xr + q);
+            if (GRAN == MOFQ_PER_GROUP) {
+                const int g = q / lanes_per_group;
+                if (scales_in) {
+                    if (active) {
+                        s = scales_in[row * gpr + g];
+                        inv = __fdiv_rn(1.0f, s);
+                    }
+                } else {
+                    uint32_t m16 = fold16(absmax_chunk(v, 0));
+                    for (int o = lanes_per_group >> 1; o; o >>= 1) m16 = max(m16, __shfl_xor_sync(0xffffffffu, m16, o));
+                    if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+                    scale_pair(mag16_to_float<DT>(m16), f.Q, s, inv, status);
+                }
+                if (scales_out && active && (q & (lanes_per_group - 1)) == 0) scales_out[row * gpr + g] = s;
+            }
+            if (!active) continue;
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            uint32_t code[8];
+            float val[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float xv[2];
+                unpack2<DT>(w[i], xv[0], xv[1]);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float t = __fmul_rn(xv[h], inv);
+                    const uint32_t neg = __float_as_uint(xv[h]) >> 31;
+                    float value;
+                    uint32_t c;
+                    if (f.is_fp) {
+                        float r = fp_grid_round(fminf(fabsf(t), 2.0f * f.Q), f.eminb, f.kadd);
+                        r = fminf(r, f.Q);
+                        c = fp_code_from_mag(r, f) | (neg << (f.bits - 1));
+                        value = neg ? -r : r;
+                    } else {
+                        float r = __fsub_rn(__fadd_rn(fminf(fmaxf(t, -1024.0f), 1024.0f), kMagic), kMagic);
+                        r = fminf(fmaxf(r, int_lo), f.Q);
+                        c = (uint32_t)((int)r) & ((1u << f.bits) - 1u);
+                        value = r;
+                    }
+                    code[2 * i + h] = c;
+                    val[2 * i + h] = value;
+                }
+            }
+            const size_t e0 = (size_t)row * cols + (size_t)q * 8;
+            if (codes_out) {
+                if (f.bits == 8) {
+                    uint2 o;
+                    o.x = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
+                    o.y = code[4] | (code[5] << 8) | (code[6] << 16) | (code[7] << 24);
+                    *reinterpret_cast<uint2 *>(codes_out + e0) = o;
+                } else {
+                    uint32_t o = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) o |= code[i] << (4 * i);
+                    *reinterpret_cast<uint32_t *>(codes_out + (e0 >> 1)) = o;
+                }
+            }
+            if (dequant_out) {
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    o[i] = (uint32_t)to_storage<DT>(__fmul_rn(val[2 * i], s)) |
+                           ((uint32_t)to_storage<DT>(__fmul_rn(val[2 * i + 1], s)) << 16);
+                *reinterpret_cast<uint4 *>(dequant_out + e0) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+            if (values_out) {  // unscaled grid values (exact in fp16 and bf16 for every format here)
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (values_dtype == MOFQ_F16)
+                        o[i] = (uint32_t)to_storage<MOFQ_F16>(val[2 * i]) | ((uint32_t)to_storage<MOFQ_F16>(val[2 * i + 1]) << 16);
+                    else
+                        o[i] = (uint32_t)to_storage<MOFQ_BF16>(val[2 * i]) | ((uint32_t)to_storage<MOFQ_BF16>(val[2 * i + 1]) << 16);
+                }
+                *reinterpret_cast<uint4 *>(values_out + e0) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+    }
+    if (status) atomicOr(&hdr->status, status);
+}
+
+// ---- host-side dispatch ----------------------------------------------------------------------------------
+#define MOFQ_CUDA_OK(expr)                      \
+    do {                                        \
+        if ((expr) != cudaSuccess) {            \
+            (void)cudaGetLastError();           \
+            return MOFQ_ERR_CUDA;               \
+        }                                       \
+    } while (0)
+
+template <typename F>
+int dispatch_cands(int dt, int ni, int nfp, F &&f)
+{
+#define MOFQ_CASE(DT_, NI_, NFP_) \
+    if (dt == DT_ && ni == NI_ && nfp == NFP_) return f(std::integral_constant<int, DT_>(), std::integral_constant<int, NI_>(), std::integral_constant<int, NFP_>());
+    MOFQ_CASE(0, 1, 0) MOFQ_CASE(0, 0, 1) MOFQ_CASE(0, 1, 1) MOFQ_CASE(0, 0, 2) MOFQ_CASE(0, 1, 2)
+    MOFQ_CASE(1, 1, 0) MOFQ_CASE(1, 0, 1) MOFQ_CASE(1, 1, 1) MOFQ_CASE(1, 0, 2) MOFQ_CASE(1, 1, 2)
+#undef MOFQ_CASE
+    return MOFQ_ERR_UNSUPPORTED;
+}
+
+int blocks_per_sm(const void *kernel, int threads, size_t smem)
+{
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+
+template <typename K>
+int set_smem(K kernel, size_t smem)
+{
+    if (smem > 48 * 1024) MOFQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    return MOFQ_OK;
+}
+
+}  // namespace
+
+int sm_count()
+{
+    static int cached = 0;
+    if (!cached) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return 148;
+        }
+        cached = n;
+    }
+    return cached;
+}
+
+int launch_score(const ScoreJob &job, cudaStream_t st)
+{
+    const mofq_tensor &x = job.x;
+    const uint16_t *xp = static_cast<const uint16_t *>(x.data);
+    const bool dense = (x.ld == x.cols);
+    const bool has_ch = job.gran == MOFQ_PER_CHANNEL || job.gran2 == MOFQ_PER_CHANNEL;
+    const bool has_grp = job.gran == MOFQ_PER_GROUP || job.gran2 == MOFQ_PER_GROUP;
+    const bool has_tensor = job.gran == MOFQ_PER_TENSOR || job.gran2 == MOFQ_PER_TENSOR;
+    const int nsm = sm_count();
+
+    if (has_tensor) {
+        if (job.gran2 != MOFQ_GRAN_NONE) return MOFQ_ERR_UNSUPPORTED;  // per-tensor cannot share a read
+        MOFQ_CUDA_OK(cudaMemsetAsync(&job.hdr->absmax_bits, 0, sizeof(uint32_t), st));
+        const long long rows = dense ? 1 : x.rows;
+        const long long cpr = dense ? x.rows * x.cols / 8 : x.cols / 8;
+        if (cpr > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+        const long long total = rows * cpr;
+        const int grid = (int)std::min<long long>((total + 255) / 256, (long long)nsm * 8);
+        if (x.dtype == MOFQ_F16)
+            kq_absmax<0><<<grid, 256, 0, st>>>(xp, rows, (int)cpr, x.ld, job.hdr);
+        else
+            kq_absmax<1><<<grid, 256, 0, st>>>(xp, rows, (int)cpr, x.ld, job.hdr);
+        MOFQ_CUDA_OK(cudaGetLastError());
+        return dispatch_cands(x.dtype, job.cs.n_int, job.cs.n_fp, [&](auto DT, auto NI, auto NFP) {
+            kq_score_uniform<DT(), NI(), NFP()><<<grid, 256, 0, st>>>(xp, rows, (int)cpr, x.ld, job.cs, job.hdr, job.partials, job.fin);
+            MOFQ_CUDA_OK(cudaGetLastError());
+            return MOFQ_OK;
+        });
+    }
+
+    if (has_grp && !has_ch && dense) {
+        const long long n_groups = x.rows * x.cols / job.group;
+        const size_t smem = (size_t)kGroupsPerTile * job.group * 2;
+        return dispatch_cands(x.dtype, job.cs.n_int, job.cs.n_fp, [&](auto DT, auto NI, auto NFP) {
+            auto kernel = kq_score_groups<DT(), NI(), NFP()>;
+            if (int rc = set_smem(kernel, smem)) return rc;
+            const int occ = std::max(1, blocks_per_sm((const void *)kernel, kGroupsPerTile, smem));
+            const long long tiles = (n_groups + kGroupsPerTile - 1) / kGroupsPerTile;
+            const int grid = (int)std::min<long long>(tiles, std::min<long long>((long long)nsm * occ, kMaxSlots));
+            kernel<<<grid, kGroupsPerTile, smem, st>>>(xp, n_groups, job.group, job.cs, job.hdr, job.partials, job.fin);
+            MOFQ_CUDA_OK(cudaGetLastError());
+            return MOFQ_OK;
+        });
+    }
+
+    // row kernel: per-channel, per-group on a strided tensor, or both from one read
+    if (x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
+    const int gpr = has_grp ? (int)(x.cols / job.group) : 0;
+    const size_t smem = (size_t)x.cols * 2 + (size_t)((gpr * 2 + 15) & ~15);
+    if (smem > 200 * 1024) return MOFQ_ERR_UNSUPPORTED;
+    const int grp_first = (job.gran == MOFQ_PER_GROUP) ? 1 : 0;
+    return dispatch_cands(x.dtype, job.cs.n_int, job.cs.n_fp, [&](auto DT, auto NI, auto NFP) {
+        auto launch = [&](auto kernel) {
+            if (int rc = set_smem(kernel, smem)) return rc;
+            const int occ = std::max(1, blocks_per_sm((const void *)kernel, kRowThreads, smem));
+            const int grid = (int)std::min<long long>(x.rows, std::min<long long>((long long)nsm * occ, kMaxSlots));
+            kernel<<<grid, kRowThreads, smem, st>>>(xp, x.rows, (int)x.cols, x.ld, has_grp ? job.group : 8, grp_first, job.cs,
+                                                    job.hdr, job.partials, job.fin);
+            MOFQ_CUDA_OK(cudaGetLastError());
+            return MOFQ_OK;
+        };
+        if (has_ch && has_grp) return launch(kq_score_rows<DT(), NI(), NFP(), true, true>);
+        if (has_ch) return launch(kq_score_rows<DT(), NI(), NFP(), true, false>);
+        return launch(kq_score_rows<DT(), NI(), NFP(), false, true>);
+    });
+}
+
+int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in, void *codes_out,
+                float *scales_out, void *dequant_out, void *values_out, int values_dtype, WsHeader *hdr, cudaStream_t st)
+{
+    const uint16_t *xp = static_cast<const uint16_t *>(x.data);
+    const int nsm = sm_count();
+    if (x.cols > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+    if (gran == MOFQ_PER_TENSOR && !scales_in) {
+        MOFQ_CUDA_OK(cudaMemsetAsync(&hdr->absmax_bits, 0, sizeof(uint32_t), st));
+        const long long total = x.rows * (x.cols / 8);
+        const int grid = (int)std::min<long long>((total + 255) / 256, (long long)nsm * 8);
+        if (x.dtype == MOFQ_F16)
+            kq_absmax<0><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, hdr);
+        else
+            kq_absmax<1><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, hdr);
+        MOFQ_CUDA_OK(cudaGetLastError());
+    }
+    const int grid = (int)std::min<long long>(x.rows, (long long)nsm * 8);
+#define MOFQ_EMIT(DT_, G_)                                                                                                   \
+    if (x.dtype == DT_ && gran == G_) {                                                                                      \
+        kq_emit<DT_, G_><<<grid, kRowThreads, 0, st>>>(xp, x.rows, (int)x.cols, x.ld, f, group, scales_in,                   \
+                                                       (unsigned char *)codes_out, scales_out, (uint16_t *)dequant_out,      \
+                                                       (uint16_t *)values_out, values_dtype, hdr);                           \
+        MOFQ_CUDA_OK(cudaGetLastError());                                                                                    \
+        return MOFQ_OK;                                                                                                      \
+    }
+    MOFQ_EMIT(0, MOFQ_PER_TENSOR) MOFQ_EMIT(0, MOFQ_PER_CHANNEL) MOFQ_EMIT(0, MOFQ_PER_GROUP)
+    MOFQ_EMIT(1, MOFQ_PER_TENSOR) MOFQ_EMIT(1, MOFQ_PER_CHANNEL) MOFQ_EMIT(1, MOFQ_PER_GROUP)
+#undef MOFQ_EMIT
+    return MOFQ_ERR_INVALID_ARG;
+}
+
+}  // namespace mofq

@@ -1,0 +1,256 @@
+"""GPU parity: quantise / score kernels against the CPU oracle, element by element (-m gpu).
+
+Bars: codes, scales, dequantised values and per-layer decisions bit-exact; MSE within 1e-5
+relative (the kernels accumulate squared errors in binary32 chains of at most 128 terms and sum
+those in double; the oracle sums in double).
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2305_12356_b200 as mofq
+from paper_2305_12356_b200 import binding as B
+from paper_2305_12356_b200 import inputs
+
+from gpu_util import host, orc_gran, rel_err, unpack_codes
+
+pytestmark = pytest.mark.gpu
+
+MSE_RTOL = 1e-5
+FMT4 = ["INT4", "FP4_E2M1", "FP4_E2M1_IEEE"]
+FMT8 = ["INT8", "FP8_E4M3", "FP8_E5M2"]
+
+
+@pytest.fixture(scope="module")
+def dev():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    mofq.lib()
+    return torch.device("cuda:0")
+
+
+def _weights(dev, rows, cols, kind="student_t", seed=1, layer=0, dtype=torch.float16, **kw):
+    w = torch.empty((rows, cols), dtype=torch.float16, device=dev)
+    inputs.device_weight(w, kind, seed, layer, **kw)
+    if dtype == torch.bfloat16:
+        w = (w.float() * 3.0).to(torch.bfloat16)
+    return w
+
+
+def _check_quantize(orc, x, name, gran, group=0, scales_in=None):
+    fmt_o = getattr(orc, name)
+    bits = orc.format_bits(fmt_o)
+    got = mofq.quantize_tensor(x, name, gran, group, scales_in=scales_in, want_dequant=True)
+    torch.cuda.synchronize()
+    xh = host(x)
+    want = orc.quantize(xh, fmt_o, orc_gran(orc, gran), group,
+                        scales_in=None if scales_in is None else scales_in.cpu().numpy(), want_dequant=True)
+    n = x.numel()
+    np.testing.assert_array_equal(unpack_codes(got["codes"], bits, n), want["codes"].reshape(-1))
+    np.testing.assert_array_equal(got["scales"].cpu().numpy().view(np.uint32), want["scales"].view(np.uint32))
+    deq = got["dequant"].cpu().view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(deq, want["dequant"])
+    assert int(got["status"].item()) == 0
+    return got, want
+
+
+# ---- quantize: every format x granularity x dtype, several tiles and a ragged tail ------------------------
+@pytest.mark.parametrize("name", FMT4 + FMT8)
+@pytest.mark.parametrize("gran,group", [("channel", 0), ("group", 128), ("group", 32), ("tensor", 0)])
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_quantize_matches_oracle(orc, dev, name, gran, group, dtype):
+    x = _weights(dev, 301, 1152, seed=11, layer=3, dtype=dtype)      # 301 rows: ragged against every tile shape
+    _check_quantize(orc, x, name, gran, group)
+
+
+@pytest.mark.parametrize("name", ["INT4", "FP4_E2M1", "INT8", "FP8_E4M3", "FP8_E5M2"])
+def test_quantize_every_finite_fp16_pattern(orc, dev, name):
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    bits = bits[(bits & 0x7C00) != 0x7C00]                            # drop Inf/NaN
+    pad = (-bits.size) % 1024
+    bits = np.concatenate([bits, np.zeros(pad, np.uint16)])
+    x = torch.from_numpy(bits.view(np.int16).copy()).view(torch.float16).reshape(-1, 1024).to(dev)
+    for gran, group in (("channel", 0), ("group", 128), ("group", 8), ("tensor", 0)):
+        _check_quantize(orc, x, name, gran, group)
+
+
+@pytest.mark.parametrize("name", ["INT8", "FP8_E4M3", "FP8_E5M2"])
+def test_quantize_every_finite_bf16_pattern_in_range(orc, dev, name):
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    e = (bits >> 7) & 0xFF
+    bits = bits[(e >= 100) & (e <= 140) | (e == 0) & ((bits & 0x7F) == 0)]   # 2^-27 .. 2^13 and +-0
+    pad = (-bits.size) % 512
+    bits = np.concatenate([bits, np.zeros(pad, np.uint16)])
+    x = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).reshape(-1, 512).to(dev)
+    for gran, group in (("channel", 0), ("group", 64), ("tensor", 0)):
+        _check_quantize(orc, x, name, gran, group)
+
+
+@pytest.mark.parametrize("name", FMT4 + FMT8)
+def test_quantize_with_supplied_scales_saturates(orc, dev, name):
+    x = _weights(dev, 40, 512, seed=12, layer=1)
+    for gran, group in (("tensor", 0), ("channel", 0), ("group", 128)):
+        ns = B.n_scales(gran, 40, 512, group)
+        g = torch.Generator().manual_seed(3)
+        scales = (torch.rand(ns, generator=g) * 0.004 + 0.0005).to(dev)      # small scales: many values clip
+        _check_quantize(orc, x, name, gran, group, scales_in=scales)
+
+
+def test_quantize_zero_rows_and_tiny_shapes(orc, dev):
+    x = _weights(dev, 9, 256, seed=13)
+    x[2].zero_()
+    x[5, :128].zero_()
+    x[7, 3] = -0.0
+    for name in ("INT4", "FP4_E2M1", "INT8", "FP8_E4M3"):
+        for gran, group in (("channel", 0), ("group", 128), ("tensor", 0)):
+            _check_quantize(orc, x, name, gran, group)
+    one = _weights(dev, 1, 8, seed=14)
+    for gran, group in (("channel", 0), ("group", 8), ("tensor", 0)):
+        _check_quantize(orc, one, "FP4_E2M1", gran, group)
+    z = torch.zeros(4, 128, dtype=torch.float16, device=dev)
+    got, _ = _check_quantize(orc, z, "INT4", "tensor")
+    assert float(got["scales"][0]) == 1.0
+
+
+def test_quantize_strided_input(orc, dev):
+    full = _weights(dev, 64, 1024, seed=15)
+    view = full[:, 256:768]                                                   # ld = 1024, cols = 512
+    got = mofq.quantize_tensor(view, "FP4_E2M1", "group", 128)
+    want = orc.quantize(host(view).contiguous(), orc.FP4_E2M1, orc.PER_GROUP, 128)
+    np.testing.assert_array_equal(unpack_codes(got["codes"], 4, view.numel()), want["codes"].reshape(-1))
+    np.testing.assert_array_equal(got["scales"].cpu().numpy(), want["scales"])
+
+
+def test_nonfinite_input_sets_status(dev):
+    x = _weights(dev, 16, 256, seed=16)
+    x[3, 7] = float("inf")
+    for gran, group in (("channel", 0), ("group", 128), ("tensor", 0)):
+        got = mofq.quantize_tensor(x, "INT4", gran, group)
+        assert int(got["status"].item()) & B.STATUS_NONFINITE_INPUT
+        _, st = mofq.tensor_error(x, ["INT4", "FP4_E2M1"], gran, group=group)
+        assert int(st.item()) & B.STATUS_NONFINITE_INPUT
+    tiny = torch.full((8, 128), 1e-38, dtype=torch.bfloat16, device=dev)     # Q / absmax overflows binary32
+    got = mofq.quantize_tensor(tiny, "FP8_E5M2", "channel")
+    assert int(got["status"].item()) & B.STATUS_SCALE_OVERFLOW
+
+
+# ---- tensor error ------------------------------------------------------------------------------------------------
+def _oracle_mse(orc, xh, names, gran, group):
+    return [orc.tensor_mse(xh, getattr(orc, n), orc_gran(orc, gran), group) for n in names]
+
+
+@pytest.mark.parametrize("names", [["INT4", "FP4_E2M1"], ["FP4_E2M1", "INT4", "FP4_E2M1_IEEE"], ["INT8", "FP8_E4M3", "FP8_E5M2"],
+                                   ["FP8_E5M2"], ["INT8"], ["FP8_E4M3", "FP8_E5M2"]])
+@pytest.mark.parametrize("gran,group", [("channel", 0), ("group", 128), ("tensor", 0)])
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_tensor_error_matches_oracle(orc, dev, names, gran, group, dtype):
+    x = _weights(dev, 333, 1408, seed=21, layer=2, dtype=dtype)               # 1408 = 11 * 128
+    got, st = mofq.tensor_error(x, names, gran, group=group)
+    want = _oracle_mse(orc, host(x), names, gran, group)
+    assert rel_err(got.cpu().numpy(), want).max() < MSE_RTOL
+    assert int(st.item()) == 0
+
+
+@pytest.mark.parametrize("kind,kw", [("gauss_outlier", {}), ("laplace", {}), ("student_t", {})])
+def test_tensor_error_two_granularities_from_one_read(orc, dev, kind, kw):
+    x = _weights(dev, 150, 6656, kind=kind, seed=22, layer=4)                 # LLaMA-33B hidden width: 52 groups per row
+    names = ["INT4", "FP4_E2M1"]
+    for g1, g2 in (("channel", "group"), ("group", "channel")):
+        got, _ = mofq.tensor_error(x, names, g1, gran2=g2, group=128)
+        want = np.array([_oracle_mse(orc, host(x), names, g1, 128), _oracle_mse(orc, host(x), names, g2, 128)])
+        assert rel_err(got.cpu().numpy(), want).max() < MSE_RTOL
+
+
+def test_tensor_error_strided_group_uses_row_kernel(orc, dev):
+    full = _weights(dev, 48, 2048, seed=23)
+    view = full[:, 512:1536]
+    got, _ = mofq.tensor_error(view, ["INT4", "FP4_E2M1"], "group", group=128)
+    want = _oracle_mse(orc, host(view).contiguous(), ["INT4", "FP4_E2M1"], "group", 128)
+    assert rel_err(got.cpu().numpy(), want).max() < MSE_RTOL
+
+
+def test_tensor_error_is_deterministic(dev):
+    x = _weights(dev, 512, 4096, seed=24)
+    for gran, group in (("channel", 0), ("group", 128), ("tensor", 0)):
+        a, _ = mofq.tensor_error(x, ["INT4", "FP4_E2M1"], gran, group=group)
+        b, _ = mofq.tensor_error(x, ["INT4", "FP4_E2M1"], gran, group=group)
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+
+
+def test_zero_tensor_and_grid_tensor(orc, dev):
+    z = torch.zeros(64, 512, dtype=torch.float16, device=dev)
+    got, _ = mofq.tensor_error(z, ["INT4", "FP4_E2M1"], "channel")
+    assert got.tolist() == [0.0, 0.0]
+    tab = orc.decode_table(orc.FP4_E2M1)
+    g = np.random.default_rng(1)
+    x = torch.from_numpy(g.choice(tab, (64, 512)) / 64.0).to(torch.float16)
+    x[:, 0] = 6.0 / 64
+    got, _ = mofq.tensor_error(x.to(dev), ["INT4", "FP4_E2M1"], "channel")
+    assert got[1].item() == 0.0 and got[0].item() > 0.0
+
+
+# ---- the single-layer workload at full size (4096 x 4096, per-channel, INT4 vs FP4) ---------------------------------
+def test_single_layer_workload_full_size(orc, dev):
+    wl = inputs.WORKLOADS["single_4096_w4_channel"]
+    w = torch.empty((4096, 4096), dtype=torch.float16, device=dev)
+    inputs.device_weight(w, wl["w_kind"], wl["seed"], 0, **wl["w_args"])
+    wh = host(w)
+    cfg = mofq.make_config(4, wl["candidates"], w_gran="channel")
+    rec = mofq.select_formats([w], cfg)[0]
+    want = [orc.tensor_mse(wh, getattr(orc, n), orc.PER_CHANNEL) for n in wl["candidates"]]
+    assert rel_err(rec["errors"], want).max() < MSE_RTOL
+    assert rec["chosen"] == orc.select(want) and rec["status"] == 0
+    for name in wl["candidates"]:
+        got = mofq.quantize_tensor(w, name, "channel")
+        ref = orc.quantize(wh, getattr(orc, name), orc.PER_CHANNEL)
+        np.testing.assert_array_equal(unpack_codes(got["codes"], 4, w.numel()), ref["codes"].reshape(-1))
+        np.testing.assert_array_equal(got["scales"].cpu().numpy().view(np.uint32), ref["scales"].view(np.uint32))
+
+
+# ---- selection over a layer list (Algorithm 1) ------------------------------------------------------------------------
+def _small_model(dev, kind, seed, shapes, **kw):
+    return [_weights(dev, o, i, kind=kind, seed=seed, layer=l, **kw) for l, (o, i) in enumerate(shapes)]
+
+
+@pytest.mark.parametrize("gran,group,gran2", [("group", 128, None), ("channel", 0, None), ("channel", 128, "group"), ("tensor", 0, None)])
+def test_select_formats_matches_oracle(orc, dev, gran, group, gran2):
+    shapes = [(256, 512), (256, 512), (688, 512), (512, 1408), (128, 128), (40, 256)]
+    layers = _small_model(dev, "student_t", 31, shapes)
+    layers[4].zero_()                                                         # tie at zero error -> first candidate
+    cands = ["INT4", "FP4_E2M1"]
+    cfg = mofq.make_config(4, cands, w_gran=gran, w_group=group, w_gran2=gran2)
+    recs = mofq.select_formats(layers, cfg)
+    n_sets = 2 if gran2 else 1
+    assert len(recs) == len(layers) * n_sets
+    for li, w in enumerate(layers):
+        for s, g in enumerate([gran, gran2][:n_sets]):
+            want = [orc.tensor_mse(host(w), getattr(orc, n), orc_gran(orc, g), 128 if g == "group" else 0) for n in cands]
+            r = recs[li * n_sets + s]
+            assert r["status"] == 0
+            if max(want) > 0:
+                assert rel_err(r["errors"], want).max() < MSE_RTOL
+            assert r["chosen"] == orc.select(want), (li, g, want, r)
+    assert recs[4 * n_sets]["chosen"] == 0 and recs[4 * n_sets]["errors"] == [0.0, 0.0]
+    swapped = mofq.make_config(4, cands[::-1], w_gran=gran, w_group=group, w_gran2=gran2)
+    recs2 = mofq.select_formats(layers, swapped)
+    assert recs2[4 * n_sets]["chosen"] == 0                                   # still the first in the caller's order
+    for a, b in zip(recs, recs2):
+        if a["errors"][0] != a["errors"][1]:
+            assert a["chosen"] == 1 - b["chosen"]
+
+
+def test_select_formats_host_buffers(orc, dev):
+    shapes = [(256, 512), (128, 1024), (64, 256)]
+    layers = [host(w).pin_memory() for w in _small_model(dev, "laplace", 32, shapes)]
+    cfg = mofq.make_config(4, ["INT4", "FP4_E2M1"], w_gran="group", w_group=128)
+    recs = mofq.select_formats_host(layers, cfg, dev)
+    for w, r in zip(layers, recs):
+        want = [orc.tensor_mse(w, f, orc.PER_GROUP, 128) for f in (orc.INT4, orc.FP4_E2M1)]
+        assert rel_err(r["errors"], want).max() < MSE_RTOL and r["chosen"] == orc.select(want)
+
+
+def test_margins_are_reported(dev):
+    layers = _small_model(dev, "student_t", 33, [(256, 512)])
+    cfg = mofq.make_config(4, ["INT4", "FP4_E2M1"], w_gran="channel")
+    r = mofq.select_formats(layers, cfg)[0]
+    e = sorted(r["errors"])
+    assert r["rel_margin"] == pytest.approx((e[1] - e[0]) / e[0], rel=1e-4)
