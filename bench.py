@@ -1,0 +1,297 @@
+#!/usr/bin/env python
+"""Throughput of MoFQ per-layer format selection on B200.
+
+A step is one whole-model selection (Algorithm 1 over every linear layer of the workload):
+quantise every weight tensor onto each candidate grid, reduce the errors, pick per layer.
+Default workload: LLaMA-7B-shaped, weight-only 4-bit, group-128 scales, INT4 vs FP4-E2M1 by
+tensor MSE, synthetic fp16 weights resident in HBM (12.95 GB, larger than L2).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` counts fp16 bytes of tensor quantised+scored per second
+over all ranks; `e2e` is the same metric through the host-buffer entry point (pinned host
+tensors, host->device copies inside the timed region); `roofline` relates the scoring kernel to
+the measured HBM copy bandwidth; `cpu_baseline` is the CPU oracle on a bounded sample.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "GB/s of fp16 tensor quantized+scored (both formats)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b_w4_group128")
+    ap.add_argument("--blocks", type=int, default=None, help="decoder blocks to build (default: the workload's)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return json.load(open(path)), "measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons for one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------------------
+def cpu_oracle_sample(workload, budget_s=12.0, max_chunks=64):
+    """Time the CPU oracle (as it stands) on chunks of the workload's first layers."""
+    from oracle import api as orc
+    from paper_2305_12356_b200 import inputs
+    wl = inputs.WORKLOADS[workload]
+    layers = inputs.workload_layers(workload)
+    cands = [getattr(orc, c) for c in wl["candidates"]]
+    grans = [{"channel": orc.PER_CHANNEL, "group": orc.PER_GROUP, "tensor": orc.PER_TENSOR}[g] for g in wl["w_gran"]]
+    orc.lib()
+    done_bytes, t_total, chunks = 0, 0.0, 0
+    while t_total < budget_s and chunks < max_chunks:
+        name, out_f, in_f = layers[chunks % len(layers)]
+        rows = min(out_f, 1024)
+        w = inputs.weight_cpu(wl["w_kind"], rows, in_f, wl["seed"], chunks % len(layers), **wl["w_args"])
+        t0 = time.perf_counter()
+        for g in grans:
+            errs = [orc.tensor_mse(w, f, g, wl["group"]) for f in cands]
+            orc.select(errs)
+        t_total += time.perf_counter() - t0
+        done_bytes += w.numel() * 2
+        chunks += 1
+    return {"value": done_bytes / t_total / 1e9, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{chunks} chunks of <=1024 rows from the first layers ({done_bytes / 1e6:.0f} MB fp16), "
+                      f"{t_total:.1f} s of CPU work, tensor-MSE criterion"}, done_bytes, t_total
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2305_12356_b200 import inputs
+    wl = inputs.WORKLOADS[args.workload]
+    times, nbytes = [], 0
+    per_step_budget = max(2.0, min(15.0, 120.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup + args.steps):
+        cb, b, t = cpu_oracle_sample(args.workload, budget_s=per_step_budget)
+        if i >= args.warmup:
+            times.append(t)
+            nbytes += b
+    value = nbytes / sum(times) / 1e9
+    cb["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "candidates": list(wl["candidates"]), "granularity": list(wl["w_gran"]),
+                   "group": wl["group"], "criterion": wl["metric"], "note": "CPU oracle on a bounded sample per step"},
+        "cpu_baseline": cb,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# --------------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2305_12356_b200 as mofq
+    from paper_2305_12356_b200 import binding as B
+    from paper_2305_12356_b200 import inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    mofq.lib()
+
+    wl = inputs.WORKLOADS[args.workload]
+    if wl["metric"] != "tensor":
+        raise SystemExit("this bench times the tensor-MSE workloads; the layer-output criterion is not built yet")
+    shapes = inputs.workload_layers(args.workload, args.blocks)
+    # weak scaling: every rank scores a whole model of its own (seed offset by rank); no data-path collective
+    seed = wl["seed"] + 1000 * rank
+    layers = []
+    for li, (_, out_f, in_f) in enumerate(shapes):
+        w = torch.empty((out_f, in_f), dtype=torch.float16, device=dev)
+        inputs.device_weight(w, wl["w_kind"], seed, li, **wl["w_args"])
+        layers.append(w)
+    n_elems = sum(w.numel() for w in layers)
+    fp16_bytes = 2 * n_elems
+    grans = wl["w_gran"]
+    cfg = mofq.make_config(wl["bits"], wl["candidates"], metric="tensor", w_gran=grans[0], w_group=wl["group"],
+                           w_gran2=grans[1] if len(grans) > 1 else None)
+    n_rec = len(layers) * len(grans)
+    results = torch.empty(n_rec * B.RESULT_BYTES, dtype=torch.uint8, device=dev)
+    ws = torch.empty(mofq.workspace_bytes(layers, cfg), dtype=torch.uint8, device=dev)
+
+    def step():
+        mofq.select_formats(layers, cfg, workspace=ws, results=results, parse=False)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * fp16_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # decisions (for the record) and a sanity check that the step produced them
+    recs = B._parse_results(bytes(results.cpu().numpy()), n_rec, cfg.n_candidates)
+    assert all(r["status"] == 0 and 0 <= r["chosen"] < cfg.n_candidates for r in recs)
+    fp_share = sum(1 for r in recs if wl["candidates"][r["chosen"]].startswith("FP")) / len(recs)
+    min_margin = min(r["rel_margin"] for r in recs)
+
+    # end to end through the host-buffer entry point (N ranks each copy their own model)
+    e2e = None
+    if not args.no_e2e:
+        host_layers = [torch.empty(w.shape, dtype=w.dtype, pin_memory=True) for w in layers]
+        for h, w in zip(host_layers, layers):
+            h.copy_(w)
+        torch.cuda.synchronize()
+        arr = B._layer_array(host_layers, require_cuda=False)
+        import ctypes as C
+        hws = torch.empty(mofq.lib().mofq_host_workspace_bytes(arr, len(host_layers), C.byref(cfg)), dtype=torch.uint8, device=dev)
+        mofq.select_formats_host(host_layers[:2], cfg, dev, workspace=hws)        # warm-up
+        barrier()
+        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            hrecs = mofq.select_formats_host(host_layers, cfg, dev, workspace=hws)
+        e1.record()
+        barrier()
+        e_ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        assert [r["chosen"] for r in hrecs] == [r["chosen"] for r in recs]
+        e2e = {"value": world * fp16_bytes / (e_ms / args.e2e_steps * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": fp16_bytes, "d2h_bytes_per_step": n_rec * B.RESULT_BYTES,
+               "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps}
+        del host_layers, hws
+
+    if rank == 0:
+        peaks, which = measured_peaks()
+        peak = float(peaks["hbm_gbs"])
+        # algorithmic bytes: 2 B per element read once (+ 4 B per 128 elements of scale state never leaves the SM)
+        launches_per_step = len(layers)
+        roofline = {"bound": "hbm", "kernel": "kq_score_*", "achieved": fp16_bytes / (ms_per_step * 1e-3) / 1e9,
+                    "peak": peak, "peak_source": f"of {which}", "unit": "GB/s",
+                    "frac": fp16_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
+                    "frac_of_nominal_8TBs": fp16_bytes / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                    "avg_launch_us": 1e3 * ms_per_step / launches_per_step,
+                    "algorithmic_bytes_per_launch": fp16_bytes / launches_per_step, "traffic": None}
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "layers": len(layers), "elements": n_elems, "fp16_GB": fp16_bytes / 1e9,
+                       "candidates": list(wl["candidates"]), "granularity": list(grans), "group": wl["group"],
+                       "criterion": "tensor_mse", "l2": "inputs larger than L2" if fp16_bytes > 2.5e8 else "inputs fit in L2",
+                       "model_select_time_ms": ms_per_step, "fp_share": fp_share, "min_rel_margin": min_margin},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * launches_per_step, "roofline": roofline,
+        }
+        if not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_oracle_sample(args.workload)[0]
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

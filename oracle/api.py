@@ -57,6 +57,8 @@ def lib():
                                              C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, f64p, f64p]
         L.orc_select.restype = C.c_int
         L.orc_select.argtypes = [f64p, C.c_int]
+        L.orc_num_threads.restype = C.c_int
+        L.orc_num_threads.argtypes = []
         L.orc_crosscheck_fp.restype = C.c_int64
         L.orc_crosscheck_fp.argtypes = [C.c_int, C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32)]
         _lib = L
@@ -94,6 +96,10 @@ def bits_to_float(bits, dt):
     for i in range(flat.size):
         of[i] = L.orc_load(_ptr(flat[i:i + 1], C.c_uint16), dt)
     return out
+
+
+def num_threads():
+    return lib().orc_num_threads()
 
 
 def format_bits(fmt):

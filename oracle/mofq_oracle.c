@@ -25,6 +25,9 @@
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 
 /* ---- enumerations (values are part of the oracle's own interface) -------------------------- */
 enum { ORC_INT4 = 0, ORC_INT8 = 1, ORC_FP4_E2M1 = 2, ORC_FP4_E2M1_IEEE = 3, ORC_FP8_E4M3 = 4, ORC_FP8_E5M2 = 5 };
@@ -441,4 +444,14 @@ int64_t orc_crosscheck_fp(int fmt, uint32_t lo_bits, uint32_t hi_bits, uint32_t 
     }
     if (first_bad) *first_bad = fb;
     return bad;
+}
+
+/* threads the OpenMP loops above will use (for reporting beside timings) */
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
 }
