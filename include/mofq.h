@@ -69,6 +69,7 @@ typedef enum { MOFQ_TENSOR_MSE = 0, MOFQ_LAYER_OUTPUT_MSE = 1 } mofq_metric;
 #define MOFQ_ERR_MISALIGNED (-3)          /* data not 16-byte aligned, or cols / ld not a multiple of 8       */
 #define MOFQ_ERR_WORKSPACE_TOO_SMALL (-4) /* workspace_bytes below the matching *_workspace_bytes() value     */
 #define MOFQ_ERR_CUDA (-5)                /* a CUDA runtime call or kernel launch failed                      */
+#define MOFQ_ERR_SCRATCH_LIMIT (-6)       /* mofq_tensor_error_noalloc: tensor beyond the built-in scratch    */
 
 /* Asynchronous status bits (device status word / mofq_result.status). */
 #define MOFQ_STATUS_NONFINITE_INPUT 1 /* an Inf or NaN was found in the input           */
@@ -177,6 +178,39 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
  */
 int mofq_select_formats_host(const mofq_layer *layers_host_data, int n_layers, const mofq_config *cfg,
                              mofq_result *results_host, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * mofq_tensor_error_noalloc - mofq_tensor_error without a caller-provided workspace.
+ * (The paper has no counterpart for this call; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that may not call cudaMalloc at the moment it wants a tensor scored - a
+ * host application that gave all device memory to its own pool at start-up, a plug-in that must
+ * not enlarge the process, a latency-critical loop where an allocation would serialise the
+ * device.  Such callers pass inputs and outputs only; the scratch that the scoring kernels need
+ * (block counters, status word, per-block partial sums) is a fixed array of
+ * MOFQ_NOALLOC_SCRATCH_BYTES bytes built into the library.  Every GPU context that loads the
+ * library carries that array until the process ends.  The call itself performs no cudaMalloc,
+ * cudaFree or other allocating call.
+ *
+ *   x, formats, n, gran, gran2, group, mse_out   exactly as for mofq_tensor_error
+ *   status_out   nullable device int32: receives the MOFQ_STATUS_* bits of this call
+ *
+ * Limits and rules:
+ *   - Tensors of more than MOFQ_NOALLOC_MAX_ELEMENTS elements, or whose scoring pass would need
+ *     more scratch than the built-in array holds, are refused with MOFQ_ERR_SCRATCH_LIMIT and
+ *     nothing is enqueued.  Use mofq_tensor_error with your own workspace for those.
+ *   - The first call on each device looks up the device address of the array (a one-time
+ *     set-up, done with that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it still holds the previous call's data when
+ *     the next call starts; each call clears the words that must start at zero.  Two calls that
+ *     can run on the GPU at the same time (different streams, or different host threads without
+ *     ordering) race on it: order them on one stream, or with events.
+ */
+#define MOFQ_NOALLOC_SCRATCH_BYTES 131328
+#define MOFQ_NOALLOC_MAX_ELEMENTS 2147483648LL /* 2^31 elements = 4 GiB of fp16/bf16 */
+int mofq_tensor_error_noalloc(const mofq_tensor *x, const int32_t *formats, int n, int gran, int gran2, int group,
+                              float *mse_out, int32_t *status_out, void *stream);
+size_t mofq_noalloc_scratch_bytes(void);
 
 /* Workspace sizes in bytes (host-side arithmetic only). */
 size_t mofq_tensor_workspace_bytes(const mofq_tensor *x);

@@ -68,6 +68,11 @@ def lib():
         L.mofq_tensor_error.restype = C.c_int
         L.mofq_tensor_error.argtypes = [C.POINTER(MofqTensor), C.POINTER(C.c_int32), C.c_int, C.c_int, C.c_int, C.c_int,
                                         vp, vp, sz, vp]
+        L.mofq_tensor_error_noalloc.restype = C.c_int
+        L.mofq_tensor_error_noalloc.argtypes = [C.POINTER(MofqTensor), C.POINTER(C.c_int32), C.c_int, C.c_int, C.c_int, C.c_int,
+                                                vp, vp, vp]
+        L.mofq_noalloc_scratch_bytes.restype = sz
+        L.mofq_noalloc_scratch_bytes.argtypes = []
         L.mofq_layer_output_error.restype = C.c_int
         L.mofq_layer_output_error.argtypes = [C.POINTER(MofqLayer), C.POINTER(MofqConfig), vp, vp, vp, sz, vp]
         for name in ("mofq_select_formats", "mofq_select_formats_host"):
@@ -192,6 +197,27 @@ def tensor_error(x, formats, gran, gran2=None, group=0, workspace=None):
     _check(L.mofq_tensor_error(C.byref(d), fm, n, _gran(gran), g2, group, out.data_ptr(), ws.data_ptr(), ws.numel(),
                                _stream(x.device)))
     return out, ws[:4].view(torch.int32)
+
+
+def tensor_error_noalloc(x, formats, gran, gran2=None, group=0, mse_out=None, status_out=None):
+    """mofq_tensor_error_noalloc: same result as tensor_error, no workspace argument.
+
+    For callers that cannot allocate device memory: pass preallocated `mse_out` (float32, n or
+    2n elements) and optionally `status_out` (int32, 1 element) and nothing is allocated here or
+    in the library.  Without them this wrapper allocates the two small outputs for convenience.
+    """
+    L = lib()
+    d = tensor_desc(x)
+    n = len(formats)
+    fm = (C.c_int32 * n)(*[_fmt(f) for f in formats])
+    g2 = _gran(gran2)
+    if mse_out is None:
+        mse_out = torch.empty((2, n) if g2 != GRAN_NONE else (n,), dtype=torch.float32, device=x.device)
+    if status_out is None:
+        status_out = torch.zeros(1, dtype=torch.int32, device=x.device)
+    _check(L.mofq_tensor_error_noalloc(C.byref(d), fm, n, _gran(gran), g2, group, mse_out.data_ptr(),
+                                       status_out.data_ptr(), _stream(x.device)))
+    return mse_out, status_out
 
 
 def layer_output_error(X, W, cfg, workspace=None):

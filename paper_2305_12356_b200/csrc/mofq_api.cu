@@ -167,6 +167,7 @@ const char *mofq_status_string(int status)
     case MOFQ_ERR_MISALIGNED: return "pointer or leading dimension not aligned";
     case MOFQ_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case MOFQ_ERR_CUDA: return "CUDA runtime error";
+    case MOFQ_ERR_SCRATCH_LIMIT: return "tensor too large for the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
     }
 }
