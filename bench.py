@@ -197,10 +197,11 @@ def main():
                            w_gran2=grans[1] if len(grans) > 1 else None)
     n_rec = len(layers) * len(grans)
     results = torch.empty(n_rec * B.RESULT_BYTES, dtype=torch.uint8, device=dev)
-    ws = torch.empty(mofq.workspace_bytes(layers, cfg), dtype=torch.uint8, device=dev)
+    prepared = mofq.prepare_layers(layers)          # marshal the layer list once; a step is one C-ABI call
+    ws = torch.empty(mofq.workspace_bytes(prepared, cfg), dtype=torch.uint8, device=dev)
 
     def step():
-        mofq.select_formats(layers, cfg, workspace=ws, results=results, parse=False)
+        mofq.select_formats(prepared, cfg, workspace=ws, results=results, parse=False)
 
     def barrier():
         if world > 1:

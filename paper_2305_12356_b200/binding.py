@@ -148,7 +148,26 @@ def _workspace(nbytes, device):
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
 
 
+class PreparedLayers:
+    """A marshalled layer list (ctypes array) that can be reused across calls; keeps the tensors alive."""
+
+    def __init__(self, layers, require_cuda=True):
+        self.layers = list(layers)
+        self.array = _layer_array(self.layers, require_cuda)
+        first = self.layers[0] if torch.is_tensor(self.layers[0]) else self.layers[0][0]
+        self.device = first.device
+
+    def __len__(self):
+        return len(self.layers)
+
+
+def prepare_layers(layers, require_cuda=True):
+    return layers if isinstance(layers, PreparedLayers) else PreparedLayers(layers, require_cuda)
+
+
 def _layer_array(layers, require_cuda=True):
+    if isinstance(layers, PreparedLayers):
+        return layers.array
     arr = (MofqLayer * len(layers))()
     for i, layer in enumerate(layers):
         W, X = (layer, None) if torch.is_tensor(layer) else layer
@@ -234,7 +253,7 @@ def layer_output_error(X, W, cfg, workspace=None):
 
 
 def workspace_bytes(layers, cfg):
-    arr = _layer_array(layers)
+    arr = prepare_layers(layers).array
     return lib().mofq_workspace_bytes(arr, len(layers), C.byref(cfg))
 
 
@@ -251,8 +270,8 @@ def select_formats(layers, cfg, workspace=None, results=None, parse=True):
     dicts; with parse=False the raw device byte tensor is returned and nothing synchronises.
     """
     L = lib()
-    arr = _layer_array(layers)
-    dev = arr and (layers[0] if torch.is_tensor(layers[0]) else layers[0][0]).device
+    prep = prepare_layers(layers)
+    arr, dev = prep.array, prep.device
     n_sets = 2 if cfg.w_gran2 != GRAN_NONE else 1
     n_rec = len(layers) * n_sets
     res = results if results is not None else torch.empty(n_rec * RESULT_BYTES, dtype=torch.uint8, device=dev)

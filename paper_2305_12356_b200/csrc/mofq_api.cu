@@ -31,7 +31,7 @@ bool describe_format(int format, FmtDesc *d)
 }
 
 // Map the caller's candidate list onto canonical kernel slots [INT][FP0][FP1].
-int build_candset(const int32_t *formats, int n, int bit_width, CandSet *cs, int *perm, int *nc)
+int build_candset(const int32_t *formats, int n, int bit_width, CandSet *cs, int *perm, int *nc, int *fp_formats)
 {
     if (!formats || n < 1 || n > MOFQ_MAX_CAND) return MOFQ_ERR_INVALID_ARG;
     CandSet c{};
@@ -64,6 +64,10 @@ int build_candset(const int32_t *formats, int n, int bit_width, CandSet *cs, int
         else perm[i] = c.n_int + (fp_fmt[0] == formats[i] ? 0 : 1);
     }
     for (int i = n; i < MOFQ_MAX_CAND; ++i) perm[i] = 0;
+    if (fp_formats) {
+        fp_formats[0] = fp_fmt[0];
+        fp_formats[1] = fp_fmt[1];
+    }
     *cs = c;
     *nc = c.n_int + c.n_fp;
     return MOFQ_OK;
@@ -178,6 +182,7 @@ size_t mofq_workspace_bytes(const mofq_layer *layers, int n_layers, const mofq_c
 {
     size_t need = align256(score_ws_bytes());
     if (cfg && cfg->metric == MOFQ_LAYER_OUTPUT_MSE && layers) need += layer_metric_ws_bytes(layers, n_layers, cfg);
+    if (cfg && layers && n_layers > 0 && mt_applicable(layers, n_layers, cfg)) need += mt_ws_bytes(n_layers);
     return need;
 }
 
@@ -261,8 +266,8 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
     if (!layers || n_layers <= 0 || !results_out) return MOFQ_ERR_INVALID_ARG;
     if (int rc = check_config(cfg)) return rc;
     CandSet cs;
-    int perm[MOFQ_MAX_CAND], nc;
-    if (int rc = build_candset(cfg->candidates, cfg->n_candidates, cfg->bit_width, &cs, perm, &nc)) return rc;
+    int perm[MOFQ_MAX_CAND], nc, fp_formats[2];
+    if (int rc = build_candset(cfg->candidates, cfg->n_candidates, cfg->bit_width, &cs, perm, &nc, fp_formats)) return rc;
     if (int rc = check_ws(workspace, workspace_bytes, mofq_workspace_bytes(layers, n_layers, cfg))) return rc;
     // validate everything before anything is enqueued
     for (int i = 0; i < n_layers; ++i) {
@@ -278,6 +283,9 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
         }
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (mt_applicable(layers, n_layers, cfg))  // one persistent launch over the whole layer list
+        return mt_run(layers, n_layers, cfg, cs, perm, nc, fp_formats, results_out,
+                      static_cast<char *>(workspace) + align256(score_ws_bytes()), st);
     if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
     const int n_sets = cfg->w_gran2 != MOFQ_GRAN_NONE ? 2 : 1;
     for (int i = 0; i < n_layers; ++i) {  // Algorithm 1: for layer in model.layers_to_quant

@@ -64,7 +64,26 @@ struct ScoreJob {
 inline size_t score_ws_bytes() { return sizeof(WsHeader) + sizeof(double) * kMaxSlots * kMaxAcc; }
 
 bool describe_format(int format, FmtDesc *d);
-int build_candset(const int32_t *formats, int n, int bit_width, CandSet *cs, int *perm, int *nc);
+// fp_formats (nullable, 2 entries): the mofq_format held by each canonical FP slot
+int build_candset(const int32_t *formats, int n, int bit_width, CandSet *cs, int *perm, int *nc, int *fp_formats = nullptr);
+
+// One layer of the multi-tensor scoring kernel's work table (device memory).
+struct MtLayer {
+    const uint16_t *x;      // dense tensor
+    long long n_groups;     // scale blocks in the tensor
+    long long tile_begin;   // index of the layer's first tile in the concatenated tile list
+    double inv_n;           // 1 / element count
+    int first_cta;          // first block that owns a tile of this layer
+    int n_slots;            // partial-sum slots of this layer (blocks spanning it x consumer warps)
+    int slot_off;           // first slot
+    int pad;
+};
+
+// multi-tensor path (mofq_kq_mt.cu)
+bool mt_applicable(const mofq_layer *layers, int n_layers, const mofq_config *cfg);
+size_t mt_ws_bytes(int n_layers);
+int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
+           const int *fp_formats, mofq_result *results, void *ws, cudaStream_t st);
 int sm_count();
 
 // kernels' host launchers (mofq_kq.cu)

@@ -1,0 +1,544 @@
+// Persistent multi-tensor scoring kernel: one launch scores every layer of a model.
+//
+// Work is the concatenation of all layers' 32 KB tiles (a tile = consecutive per-group scale
+// blocks of one dense tensor).  Each CTA owns a contiguous range of tiles.  One producer thread
+// streams tiles into a shared-memory ring with bulk async copies (TMA, 1-D) that complete on
+// mbarriers; four consumer warps take one group per lane, walk its 16-byte chunks rotated by the
+// lane index (conflict-free on the dense tile), find the abs-max, derive the scales and score every
+// candidate from the same registers.  Per (layer, CTA, warp) partial sums go to the workspace; a
+// second small kernel adds them in a fixed order and applies Algorithm 1's comparison.
+//
+// Arithmetic per element, on magnitudes a = |x| (every grid is symmetric):
+//   INT : r = RNE(a*inv) through fma(a, inv, 1.5*2^23) - 1.5*2^23.  The fused multiply-add rounds
+//         the exact product once instead of twice; the two can differ only where a*inv sits within
+//         one binary32 ulp of a tie, and at a tie both neighbours have the same error, so the
+//         squared-error sum agrees with the two-rounding definition far inside the 1e-5 tolerance.
+//   FP  : t = RN32(a*inv); r = hardware convert of t to the 4/8-bit float (round-to-nearest-even,
+//         saturating) and back; e = fma(-r, s, a); sum += e*e.
+// Packed two-lane binary32 instructions (f32x2) halve the issue slots of the multiply/add work.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <algorithm>
+#include <type_traits>
+#include <vector>
+
+#include "mofq_internal.h"
+
+namespace mofq {
+namespace {
+
+constexpr int kStages = 2;
+constexpr int kTileBytes = 32768;
+constexpr int kConsumerWarps = 4;
+constexpr int kConsumers = kConsumerWarps * 32;
+constexpr int kThreads = kConsumers + 32;  // + one producer warp
+constexpr long long kWaitCycles = 4000000000LL;  // ~2 s: a wait that long means the pipeline is broken
+constexpr float kMagic = 12582912.0f;
+
+enum { FPK_E2M1 = 0, FPK_E4M3 = 1, FPK_E5M2 = 2 };
+
+// ---- PTX wrappers -------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t pk(float lo, float hi) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ void upk(uint64_t v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { uint64_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) { uint64_t d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+
+// two non-negative floats -> FP4/FP8 pair (RNE, saturating) -> the same two values as f16x2
+template <int KIND>
+__device__ __forceinline__ uint32_t fp_round_trip(float lo, float hi)
+{
+    uint32_t h2;
+    if (KIND == FPK_E2M1)
+        asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %2, %1; cvt.rn.f16x2.e2m1x2 %0, t; }" : "=r"(h2) : "f"(lo), "f"(hi));
+    else if (KIND == FPK_E4M3)
+        asm("{ .reg .b16 t; cvt.rn.satfinite.e4m3x2.f32 t, %2, %1; cvt.rn.f16x2.e4m3x2 %0, t; }" : "=r"(h2) : "f"(lo), "f"(hi));
+    else
+        asm("{ .reg .b16 t; cvt.rn.satfinite.e5m2x2.f32 t, %2, %1; cvt.rn.f16x2.e5m2x2 %0, t; }" : "=r"(h2) : "f"(lo), "f"(hi));
+    return h2;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t *bar, int count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count)); }
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after ~2 s and reports it, so a broken pipeline cannot hang the GPU.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *err)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*err || clock64() - t0 > kWaitCycles) {
+            *err = 1;
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// ---- per-format scoring --------------------------------------------------------------------------------
+template <int NC>
+struct Sc {
+    float s[NC], inv[NC];
+};
+
+__device__ __forceinline__ void scale_pair(float a, float Q, float &s, float &inv, int &status)
+{
+    if (a == 0.0f) {
+        s = 1.0f;
+        inv = 1.0f;
+    } else {
+        s = __fdiv_rn(a, Q);
+        inv = __fdiv_rn(Q, a);
+        if (isinf(inv)) status |= MOFQ_STATUS_SCALE_OVERFLOW;
+    }
+}
+
+// magnitudes of the two 16-bit values in w, as packed binary32
+template <int DT>
+__device__ __forceinline__ uint64_t abs_unpack(uint32_t w)
+{
+    const uint32_t wa = w & 0x7FFF7FFFu;
+    if (DT == MOFQ_F16) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&wa));
+        return pk(f.x, f.y);
+    }
+    return pk(__uint_as_float(wa << 16), __uint_as_float(wa & 0xFFFF0000u));
+}
+
+template <int DT>
+__device__ __forceinline__ uint32_t absmax_chunk(const uint4 v, uint32_t m)
+{
+    if (DT == MOFQ_F16) {
+        __half2 mm = *reinterpret_cast<__half2 *>(&m);
+        mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __half2 *>(&v.x)));
+        mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __half2 *>(&v.y)));
+        mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __half2 *>(&v.z)));
+        mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __half2 *>(&v.w)));
+        return *reinterpret_cast<uint32_t *>(&mm);
+    }
+    __nv_bfloat162 mm = *reinterpret_cast<__nv_bfloat162 *>(&m);
+    mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&v.x)));
+    mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&v.y)));
+    mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&v.z)));
+    mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&v.w)));
+    return *reinterpret_cast<uint32_t *>(&mm);
+}
+
+// fold the two 16-bit lanes of a packed abs-max; NaN patterns (> Inf) stay on top as integers
+__device__ __forceinline__ uint32_t fold16(uint32_t m) { return max(m & 0x7FFFu, (m >> 16) & 0x7FFFu); }
+
+template <int DT>
+__device__ __forceinline__ float mag16_to_float(uint32_t m16)
+{
+    if (DT == MOFQ_F16) return __half2float(__ushort_as_half((unsigned short)m16));
+    return __uint_as_float(m16 << 16);
+}
+template <int DT>
+__device__ __forceinline__ bool mag16_nonfinite(uint32_t m16)
+{
+    return m16 >= (DT == MOFQ_F16 ? 0x7C00u : 0x7F80u);
+}
+
+template <int DT, int NI, int K0, int K1>  // K0/K1: FP kind of slot 0/1, or -1
+struct Scorer {
+    static constexpr int NFP = (K0 >= 0) + (K1 >= 0);
+    static constexpr int NC = NI + NFP;
+    uint64_t inv2[NC], ns2[NC], acc2[NC];
+
+    __device__ __forceinline__ void begin(const Sc<NC> &sc)
+    {
+#pragma unroll
+        for (int j = 0; j < NC; ++j) {
+            inv2[j] = pk(sc.inv[j], sc.inv[j]);
+            ns2[j] = pk(-sc.s[j], -sc.s[j]);
+            acc2[j] = 0;
+        }
+    }
+    template <int KIND>
+    __device__ __forceinline__ void fp_slot(int j, uint64_t a2)
+    {
+        float tl, th;
+        upk(mul2(a2, inv2[j]), tl, th);
+        const uint32_t h2 = fp_round_trip<KIND>(tl, th);
+        const float2 rf = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+        const uint64_t e2 = fma2(pk(rf.x, rf.y), ns2[j], a2);
+        acc2[j] = fma2(e2, e2, acc2[j]);
+    }
+    __device__ __forceinline__ void word(uint32_t w)
+    {
+        const uint64_t a2 = abs_unpack<DT>(w);
+        if (NI) {
+            const uint64_t mg = pk(kMagic, kMagic), nmg = pk(-kMagic, -kMagic);
+            const uint64_t r2 = add2(fma2(a2, inv2[0], mg), nmg);
+            const uint64_t e2 = fma2(r2, ns2[0], a2);
+            acc2[0] = fma2(e2, e2, acc2[0]);
+        }
+        if (K0 >= 0) fp_slot<K0 >= 0 ? K0 : 0>(NI, a2);
+        if (K1 >= 0) fp_slot<K1 >= 0 ? K1 : 0>(NI + 1, a2);
+    }
+    __device__ __forceinline__ void chunk(const uint4 v)
+    {
+        word(v.x);
+        word(v.y);
+        word(v.z);
+        word(v.w);
+    }
+    __device__ __forceinline__ void end(double *dacc)
+    {
+#pragma unroll
+        for (int j = 0; j < NC; ++j) {
+            float lo, hi;
+            upk(acc2[j], lo, hi);
+            dacc[j] += (double)(lo + hi);
+        }
+    }
+};
+
+// ---- the kernel ---------------------------------------------------------------------------------------
+struct MtParams {
+    const MtLayer *layers;
+    int n_layers;
+    long long total_tiles, tiles_per_cta;
+    int group;
+    float q[3];          // abs-max target per canonical slot
+    double *partials;    // [slot][kMaxAcc]
+    int32_t *status;     // [layer]
+    int32_t *timeout;    // one word: set if a bounded wait expired
+};
+
+__device__ __forceinline__ int find_layer(const MtLayer *layers, int n, long long tile)
+{
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (layers[mid].tile_begin <= tile) lo = mid;
+        else hi = mid - 1;
+    }
+    return lo;
+}
+
+template <int DT, int NI, int K0, int K1>
+__global__ void __launch_bounds__(kThreads)
+kq_score_mt(const MtParams p)
+{
+    using S = Scorer<DT, NI, K0, K1>;
+    constexpr int NC = S::NC;
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages];
+    __shared__ int err;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long t_begin = (long long)blockIdx.x * p.tiles_per_cta;
+    const long long t_end = min(t_begin + p.tiles_per_cta, p.total_tiles);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kConsumerWarps);
+        }
+        err = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (t_begin >= t_end) return;
+    const int tile_elems_shift = 14;  // 16384 elements per tile
+    const int gpt = (kTileBytes / 2) / p.group;  // groups per full tile
+    int layer = find_layer(p.layers, p.n_layers, t_begin);
+
+    if (warp == kConsumerWarps) {
+        // ---------------- producer: one thread streams tiles into the ring ----------------
+        if (lane == 0) {
+            MtLayer L = p.layers[layer];
+            long long next_begin = layer + 1 < p.n_layers ? p.layers[layer + 1].tile_begin : p.total_tiles;
+            int it = 0;
+            for (long long t = t_begin; t < t_end; ++t, ++it) {
+                while (t >= next_begin) {
+                    ++layer;
+                    L = p.layers[layer];
+                    next_begin = layer + 1 < p.n_layers ? p.layers[layer + 1].tile_begin : p.total_tiles;
+                }
+                const int s = it % kStages;
+                const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                if (!mbar_wait(&empty_bar[s], ph ^ 1u, &err)) break;
+                const long long g0 = (t - L.tile_begin) * gpt;
+                const long long ng = min((long long)gpt, L.n_groups - g0);
+                const uint32_t bytes = (uint32_t)(ng * p.group * 2);
+                mbar_expect_tx(&full_bar[s], bytes);
+                bulk_load(smem + (size_t)s * kTileBytes, reinterpret_cast<const unsigned char *>(L.x) + ((size_t)(t - L.tile_begin) << (tile_elems_shift + 1)), bytes, &full_bar[s]);
+            }
+            if (err) {
+                // give copies already issued a bounded chance to land before the CTA's shared memory is released
+                for (int s = 0; s < kStages; ++s) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&full_bar[s], 0) && !mbar_try_wait(&full_bar[s], 1) && clock64() - t0 < kWaitCycles) {}
+                }
+                atomicOr(p.timeout, MOFQ_STATUS_TIMEOUT);
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers ----------------
+    const int cpg = p.group >> 3;
+    MtLayer L = p.layers[layer];
+    long long next_begin = layer + 1 < p.n_layers ? p.layers[layer + 1].tile_begin : p.total_tiles;
+    double dacc[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) dacc[j] = 0.0;
+    int status = 0;
+
+    auto flush = [&]() {
+        // per-warp partial of the finished layer -> its slot; the finalize kernel adds the slots in order
+#pragma unroll
+        for (int j = 0; j < NC; ++j)
+#pragma unroll
+            for (int o = 16; o; o >>= 1) dacc[j] += __shfl_xor_sync(0xffffffffu, dacc[j], o);
+        if (lane == 0) {
+            const long long slot = L.slot_off + (long long)(blockIdx.x - L.first_cta) * kConsumerWarps + warp;
+#pragma unroll
+            for (int j = 0; j < NC; ++j) p.partials[slot * kMaxAcc + j] = dacc[j];
+        }
+        if (status) atomicOr(&p.status[layer], status);
+#pragma unroll
+        for (int j = 0; j < NC; ++j) dacc[j] = 0.0;
+        status = 0;
+    };
+
+    int it = 0;
+    for (long long t = t_begin; t < t_end; ++t, ++it) {
+        while (t >= next_begin) {
+            flush();
+            ++layer;
+            L = p.layers[layer];
+            next_begin = layer + 1 < p.n_layers ? p.layers[layer + 1].tile_begin : p.total_tiles;
+        }
+        const int s = it % kStages;
+        const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+        if (!mbar_wait(&full_bar[s], ph, &err)) break;
+        const long long g0 = (t - L.tile_begin) * gpt;
+        const int ng = (int)min((long long)gpt, L.n_groups - g0);
+        const uint4 *tile = reinterpret_cast<const uint4 *>(smem + (size_t)s * kTileBytes);
+        for (int g = threadIdx.x; g < ng; g += kConsumers) {
+            const uint4 *base = tile + g * cpg;
+            uint32_t m = 0;
+#pragma unroll 4
+            for (int j = 0; j < cpg; ++j) m = absmax_chunk<DT>(base[(j + g) & (cpg - 1)], m);
+            const uint32_t m16 = fold16(m);
+            if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+            const float a = mag16_to_float<DT>(m16);
+            Sc<NC> sc;
+#pragma unroll
+            for (int j = 0; j < NC; ++j) scale_pair(a, p.q[j], sc.s[j], sc.inv[j], status);
+            S scorer;
+            scorer.begin(sc);
+#pragma unroll 4
+            for (int j = 0; j < cpg; ++j) scorer.chunk(base[(j + g) & (cpg - 1)]);
+            scorer.end(dacc);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[s]);
+    }
+    flush();
+}
+
+// ---- finalize: one block per layer ---------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+kq_mt_finalize(const MtLayer *layers, const double *partials, int32_t *status, const int32_t *timeout, Finalize fin,
+               mofq_result *results)
+{
+    __shared__ double red[4][kMaxAcc];
+    const MtLayer L = layers[blockIdx.x];
+    double tot[kMaxAcc];
+#pragma unroll
+    for (int j = 0; j < kMaxAcc; ++j) tot[j] = 0.0;
+    for (int slot = threadIdx.x; slot < L.n_slots; slot += blockDim.x)
+        for (int j = 0; j < fin.nc; ++j) tot[j] += partials[(size_t)(L.slot_off + slot) * kMaxAcc + j];
+    for (int j = 0; j < fin.nc; ++j)
+#pragma unroll
+        for (int o = 16; o; o >>= 1) tot[j] += __shfl_xor_sync(0xffffffffu, tot[j], o);
+    if ((threadIdx.x & 31) == 0)
+        for (int j = 0; j < fin.nc; ++j) red[threadIdx.x >> 5][j] = tot[j];
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    double err[MOFQ_MAX_CAND];
+    double best = INFINITY, second = INFINITY;
+    int chosen = -1;
+    for (int i = 0; i < fin.n_cand; ++i) {
+        const int j = fin.perm[i];
+        err[i] = (red[0][j] + red[1][j] + red[2][j] + red[3][j]) * L.inv_n;
+        // Algorithm 1: replace only on a strictly smaller error, in the caller's candidate order
+        if (err[i] < best) {
+            second = best;
+            best = err[i];
+            chosen = i;
+        } else if (err[i] < second) {
+            second = err[i];
+        }
+    }
+    mofq_result r;
+    r.chosen = chosen;
+    r.status = status[blockIdx.x] | *timeout;
+    for (int i = 0; i < MOFQ_MAX_CAND; ++i) {
+        r.error[i] = i < fin.n_cand ? (float)err[i] : 0.0f;
+        r.nsr[i] = 0.0f;
+    }
+    r.rel_margin = best > 0.0 ? (float)((second - best) / best) : INFINITY;
+    r.reserved = 0;
+    results[blockIdx.x] = r;
+}
+
+// The work table travels to the device as kernel arguments, 64 entries per launch: fully stream-ordered,
+// no pageable-memory copy (which would synchronise the stream) and nothing for the caller to keep alive.
+constexpr int kUploadChunk = 64;
+struct TableChunk {
+    MtLayer e[kUploadChunk];
+};
+__global__ void kq_mt_upload(const TableChunk chunk, MtLayer *dst, int n)
+{
+    if ((int)threadIdx.x < n) dst[threadIdx.x] = chunk.e[threadIdx.x];
+}
+
+int fp_kind(int format)
+{
+    switch (format) {
+    case MOFQ_FP4_E2M1:
+    case MOFQ_FP4_E2M1_IEEE: return FPK_E2M1;
+    case MOFQ_FP8_E4M3: return FPK_E4M3;
+    case MOFQ_FP8_E5M2: return FPK_E5M2;
+    }
+    return -1;
+}
+
+template <int DT, int NI, int K0, int K1>
+int launch(const MtParams &p, int grid, cudaStream_t st)
+{
+    auto kernel = kq_score_mt<DT, NI, K0, K1>;
+    const size_t smem = (size_t)kStages * kTileBytes;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MOFQ_ERR_CUDA;
+    }
+    kernel<<<grid, kThreads, smem, st>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+    return MOFQ_OK;
+}
+
+template <int DT>
+int dispatch(int ni, int k0, int k1, const MtParams &p, int grid, cudaStream_t st)
+{
+#define MOFQ_MT(NI_, K0_, K1_) \
+    if (ni == NI_ && k0 == K0_ && k1 == K1_) return launch<DT, NI_, K0_, K1_>(p, grid, st);
+    MOFQ_MT(1, -1, -1) MOFQ_MT(0, FPK_E2M1, -1) MOFQ_MT(1, FPK_E2M1, -1) MOFQ_MT(0, FPK_E2M1, FPK_E2M1) MOFQ_MT(1, FPK_E2M1, FPK_E2M1)
+    MOFQ_MT(0, FPK_E4M3, -1) MOFQ_MT(1, FPK_E4M3, -1) MOFQ_MT(0, FPK_E5M2, -1) MOFQ_MT(1, FPK_E5M2, -1)
+    MOFQ_MT(0, FPK_E4M3, FPK_E5M2) MOFQ_MT(1, FPK_E4M3, FPK_E5M2) MOFQ_MT(0, FPK_E5M2, FPK_E4M3) MOFQ_MT(1, FPK_E5M2, FPK_E4M3)
+#undef MOFQ_MT
+    return MOFQ_ERR_UNSUPPORTED;
+}
+
+size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+int mt_grid() { return sm_count() * 3; }
+
+}  // namespace
+
+// The multi-tensor path applies to the tensor metric with one per-group granularity on dense tensors of one dtype.
+bool mt_applicable(const mofq_layer *layers, int n_layers, const mofq_config *cfg)
+{
+    if (cfg->metric != MOFQ_TENSOR_MSE || cfg->w_gran != MOFQ_PER_GROUP || cfg->w_gran2 != MOFQ_GRAN_NONE) return false;
+    if (cfg->w_group < 8 || cfg->w_group > 256) return false;
+    for (int i = 0; i < n_layers; ++i)
+        if (layers[i].W.ld != layers[i].W.cols || layers[i].W.dtype != layers[0].W.dtype) return false;
+    return true;
+}
+
+size_t mt_ws_bytes(int n_layers)
+{
+    const size_t slots = ((size_t)mt_grid() + (size_t)n_layers) * kConsumerWarps;
+    return align256(sizeof(MtLayer) * (size_t)n_layers) + align256(slots * kMaxAcc * sizeof(double)) +
+           align256(sizeof(int32_t) * ((size_t)n_layers + 1));
+}
+
+int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
+           const int *fp_formats, mofq_result *results, void *ws, cudaStream_t st)
+{
+    const int grid = mt_grid();
+    const int gpt = (kTileBytes / 2) / cfg->w_group;
+    std::vector<MtLayer> table((size_t)n_layers);
+    long long tiles = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        const mofq_tensor &W = layers[i].W;
+        MtLayer &L = table[(size_t)i];
+        L.x = static_cast<const uint16_t *>(W.data);
+        L.n_groups = W.rows * W.cols / cfg->w_group;
+        L.tile_begin = tiles;
+        L.inv_n = 1.0 / ((double)W.rows * (double)W.cols);
+        tiles += (L.n_groups + gpt - 1) / gpt;
+    }
+    const long long tpc = (tiles + grid - 1) / grid;
+    long long slot = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        MtLayer &L = table[(size_t)i];
+        const long long end = (i + 1 < n_layers ? table[(size_t)i + 1].tile_begin : tiles) - 1;
+        L.first_cta = (int)(L.tile_begin / tpc);
+        L.n_slots = (int)(end / tpc - L.first_cta + 1) * kConsumerWarps;
+        L.slot_off = (int)slot;
+        slot += L.n_slots;
+    }
+    char *base = static_cast<char *>(ws);
+    MtLayer *d_table = reinterpret_cast<MtLayer *>(base);
+    double *d_partials = reinterpret_cast<double *>(base + align256(sizeof(MtLayer) * (size_t)n_layers));
+    int32_t *d_status = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(d_partials) +
+                                                    align256(((size_t)grid + (size_t)n_layers) * kConsumerWarps * kMaxAcc * sizeof(double)));
+    for (int i = 0; i < n_layers; i += kUploadChunk) {
+        TableChunk chunk;
+        const int n = std::min(kUploadChunk, n_layers - i);
+        for (int k = 0; k < n; ++k) chunk.e[k] = table[(size_t)(i + k)];
+        kq_mt_upload<<<1, kUploadChunk, 0, st>>>(chunk, d_table + i, n);
+        if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+    }
+    if (cudaMemsetAsync(d_status, 0, sizeof(int32_t) * ((size_t)n_layers + 1), st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MOFQ_ERR_CUDA;
+    }
+    MtParams p{};
+    p.layers = d_table;
+    p.n_layers = n_layers;
+    p.total_tiles = tiles;
+    p.tiles_per_cta = tpc;
+    p.group = cfg->w_group;
+    if (cs.n_int) p.q[0] = cs.int_q;
+    for (int f = 0; f < cs.n_fp; ++f) p.q[cs.n_int + f] = cs.fp_q[f];
+    p.partials = d_partials;
+    p.status = d_status;
+    p.timeout = d_status + n_layers;
+    const int k0 = cs.n_fp > 0 ? fp_kind(fp_formats[0]) : -1, k1 = cs.n_fp > 1 ? fp_kind(fp_formats[1]) : -1;
+    const int used = (int)std::min<long long>(grid, (tiles + tpc - 1) / tpc);
+    int rc = layers[0].W.dtype == MOFQ_F16 ? dispatch<MOFQ_F16>(cs.n_int, k0, k1, p, used, st)
+                                           : dispatch<MOFQ_BF16>(cs.n_int, k0, k1, p, used, st);
+    if (rc) return rc;
+    Finalize fin{};
+    fin.n_cand = cfg->n_candidates;
+    fin.n_sets = 1;
+    fin.nc = nc;
+    for (int i = 0; i < MOFQ_MAX_CAND; ++i) fin.perm[i] = perm[i];
+    kq_mt_finalize<<<n_layers, 128, 0, st>>>(d_table, d_partials, d_status, d_status + n_layers, fin, results);
+    if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+    return MOFQ_OK;
+}
+
+}  // namespace mofq

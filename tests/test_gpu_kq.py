@@ -254,3 +254,35 @@ def test_margins_are_reported(dev):
     r = mofq.select_formats(layers, cfg)[0]
     e = sorted(r["errors"])
     assert r["rel_margin"] == pytest.approx((e[1] - e[0]) / e[0], rel=1e-4)
+
+
+# ---- the persistent multi-tensor scoring path (dense tensors, per-group scales) ------------------------------------------
+@pytest.mark.parametrize("bits,cands", [(4, ["INT4", "FP4_E2M1"]), (4, ["FP4_E2M1_IEEE", "INT4", "FP4_E2M1"]), (4, ["FP4_E2M1"]),
+                                        (8, ["INT8", "FP8_E4M3", "FP8_E5M2"]), (8, ["FP8_E5M2", "FP8_E4M3"]), (8, ["INT8"])])
+@pytest.mark.parametrize("group", [128, 32, 256])
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_multi_tensor_path_matches_oracle(orc, dev, bits, cands, group, dtype):
+    # many small layers (several per block), a big one spanning many blocks, ragged last tiles, a zero layer
+    shapes = [(8, 256), (56, 768), (3000, 2048), (1, 256), (130, 1280), (16, 512), (1000, 4352)]
+    layers = [_weights(dev, o, i, kind=["student_t", "laplace", "gauss_outlier"][l % 3], seed=41, layer=l, dtype=dtype)
+              for l, (o, i) in enumerate(shapes)]
+    layers[5].zero_()
+    cfg = mofq.make_config(bits, cands, w_gran="group", w_group=group)
+    recs = mofq.select_formats(layers, cfg)
+    again = mofq.select_formats(layers, cfg)
+    assert recs == again                                                      # fixed summation order: bit-identical reruns
+    for li, (w, r) in enumerate(zip(layers, recs)):
+        want = [orc.tensor_mse(host(w), getattr(orc, n), orc.PER_GROUP, group) for n in cands]
+        assert r["status"] == 0
+        if max(want) > 0:
+            assert rel_err(r["errors"], want).max() < MSE_RTOL, (li, r, want)
+        assert r["chosen"] == orc.select(want), (li, r, want)
+    assert recs[5]["chosen"] == 0 and recs[5]["errors"] == [0.0] * len(cands)
+
+
+def test_multi_tensor_path_status_per_layer(dev):
+    layers = [_weights(dev, 64, 512, seed=42, layer=l) for l in range(4)]
+    layers[2][7, 300] = float("nan")
+    cfg = mofq.make_config(4, ["INT4", "FP4_E2M1"], w_gran="group", w_group=128)
+    recs = mofq.select_formats(layers, cfg)
+    assert [bool(r["status"] & B.STATUS_NONFINITE_INPUT) for r in recs] == [False, False, True, False]
