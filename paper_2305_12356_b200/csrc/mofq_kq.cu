@@ -631,6 +631,21 @@ int sm_count()
     return cached;
 }
 
+// abs-max of the whole tensor into hdr->absmax_bits (the caller has cleared that word)
+int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st)
+{
+    if (x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+    const uint16_t *xp = static_cast<const uint16_t *>(x.data);
+    const long long total = x.rows * (x.cols / 8);
+    const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
+    if (x.dtype == MOFQ_F16)
+        kq_absmax<0><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, hdr);
+    else
+        kq_absmax<1><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, hdr);
+    MOFQ_CUDA_OK(cudaGetLastError());
+    return MOFQ_OK;
+}
+
 int launch_score(const ScoreJob &job, cudaStream_t st)
 {
     const mofq_tensor &x = job.x;

@@ -1,13 +1,546 @@
-// Layer-output metric: Y = X W^T against its quantised counterparts (Section 3.2, layer analysis).
+// Layer-output metric (Section 3.2, layer analysis): error of Y = X W^T when W (and X) are quantised.
+//
+//   reference pass : Y[t,o] = sum_i X[t,i] W[o,i]            (fp32 accumulation of the exact operands), sum Y^2
+//   per format f   : Yq = a_f * s_w[o] * (A_f B_f^T),  sum (Y - Yq)^2
+//                    WA     : A_f = grid values of X, B_f = grid values of W, a_f = s_x
+//                    W-only : A_f = X,                B_f = grid values of W, a_f = 1
+// The grid values of INT8 / E4M3 / E5M2 / INT4 / E2M1 are exactly representable in fp16 and bf16, so every
+// product below is exact and only the fp32 accumulation rounds.
+//
+// One GEMM kernel serves all passes: tcgen05.mma (kind::f16, M=128, N=128, K=16) issued by one
+// thread, operands staged by TMA (128-byte swizzle, K-major, no multicast) through a 6-stage
+// shared-memory ring, two 128-column fp32 accumulators in tensor memory so that the epilogue of one
+// tile overlaps the main loop of the next.  The epilogue reads the accumulator with tcgen05.ld,
+// applies the scales, forms Y (stored once, fp32) or the difference to the stored Y, and reduces the
+// squares; per-CTA partial sums are added in a fixed order by a small finalize kernel.
+// Every mbarrier wait is bounded: on expiry the CTA records MOFQ_STATUS_TIMEOUT, frees its tensor
+// memory and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <algorithm>
+
 #include "mofq_internal.h"
 
 namespace mofq {
+namespace {
 
-size_t layer_metric_ws_bytes(const mofq_layer *, int, const mofq_config *) { return 0; }
+constexpr int BM = 128, BN = 128, BK = 64;
+constexpr int kStages = 6;
+constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2;
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kGemmThreads = 192;  // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-5: epilogue
+constexpr int kTmemCols = 256;     // two accumulators of BN columns
+constexpr long long kWaitCycles = 4000000000LL;
+constexpr int kMaxGemmCtas = 148 * 2;
 
-int layer_metric_run(const mofq_layer &, const mofq_config *, mofq_result *, float *, float *, void *, size_t, cudaStream_t)
+// ---- PTX wrappers ----------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t *bar, int count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count)); }
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
 {
-    return MOFQ_ERR_UNSUPPORTED;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *err)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*err || clock64() - t0 > kWaitCycles) {
+            *err = 1;
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i receives row (lane base + i)
+__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+                   "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+                   "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+                   "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor for a K-major tile whose rows are 128 bytes (64 16-bit elements) written
+// by TMA with the 128-byte swizzle: 8-row atoms of 1024 bytes, stacked along M/N.
+__device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) /* leading offset: unused with a swizzle */ |
+           ((uint64_t)(1024 >> 4) << 32) /* stride between 8-row atoms */ | (1ull << 46) /* descriptor version */ |
+           (2ull << 61) /* 128-byte swizzle */;
+}
+
+struct GemmParams {
+    int M, N, K;              // Y is M x N, contraction over K
+    int mode;                 // 0: reference (write Y, sum Y^2); 1: quantised (sum (Y - alpha*col*acc)^2)
+    float *Y;                 // [M, N] fp32, dense
+    const float *alpha;       // device scalar
+    const float *col_scale;   // device [N] or nullptr (treated as 1)
+    double *partials;         // one double per CTA
+    int32_t *status;          // device status word (timeout)
+    uint32_t idesc;
+};
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], tfull_bar[2], tempty_bar[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int err_flag;
+    __shared__ double red[4];
+    volatile int *const perr = &err_flag;
+#define err (*perr)
+
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+    const int n_tiles = tiles_m * tiles_n;
+    const int kblocks = (p.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&tfull_bar[b], 1);
+            mbar_init(&tempty_bar[b], 4);
+        }
+        err = 0;
+        red[0] = red[1] = red[2] = red[3] = 0.0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {  // the MMA warp owns the tensor-memory allocation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&tmem_base_slot);
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int it = 0;
+            for (int tile = blockIdx.x; tile < n_tiles && !err; tile += gridDim.x) {
+                const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    if (!mbar_wait(&empty_bar[s], ((it / kStages) & 1) ^ 1, perr)) break;
+                    mbar_expect_tx(&full_bar[s], kStageBytes);
+                    unsigned char *st = smem + (size_t)s * kStageBytes;
+                    tma_load_2d(st, &map_a, kb * BK, m0, &full_bar[s]);
+                    tma_load_2d(st + kABytes, &map_b, kb * BK, n0, &full_bar[s]);
+                }
+            }
+            if (err) {  // let copies that are still in flight land before the shared memory is given back
+                for (int s = 0; s < kStages; ++s) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&full_bar[s], 0) && !mbar_try_wait(&full_bar[s], 1) && clock64() - t0 < kWaitCycles) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            int it = 0, local = 0;
+            for (int tile = blockIdx.x; tile < n_tiles && !err; tile += gridDim.x, ++local) {
+                const int buf = local & 1;
+                if (!mbar_wait(&tempty_bar[buf], ((local >> 1) & 1) ^ 1, perr)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                bool ok = true;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    if (!mbar_wait(&full_bar[s], (it / kStages) & 1, perr)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
+                    const uint64_t a_desc = smem_desc_k_major_sw128(sa), b_desc = smem_desc_k_major_sw128(sa + kABytes);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)  // each step advances 16 elements = 32 bytes inside the swizzled row
+                        tc_mma_f16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc, (kb | k) != 0);
+                    tc_commit(&empty_bar[s]);  // the stage is free once these MMAs have read it
+                }
+                if (!ok) break;
+                tc_commit(&tfull_bar[buf]);    // accumulator complete
+            }
+        }
+    } else {
+        // ---------------- epilogue: warps 2..5 read the lane quarter (warp % 4) of the accumulator ----------------
+        const int q = warp & 3;
+        const float alpha = *p.alpha;
+        double dsum = 0.0;
+        int local = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++local) {
+            const int buf = local & 1;
+            const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+            if (!mbar_wait(&tfull_bar[buf], (local >> 1) & 1, perr)) break;
+            tc_fence_after();
+            const int row = m0 + q * 32 + lane;
+            float fsum = 0.0f;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), r);
+                const int col0 = n0 + c * 32;
+                if (row < p.M) {
+                    float *yrow = p.Y + (size_t)row * p.N + col0;
+                    if (col0 + 32 <= p.N && (p.N & 3) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            float4 v;
+                            if (p.mode == 0) {
+                                v.x = __uint_as_float(r[j]) * alpha;
+                                v.y = __uint_as_float(r[j + 1]) * alpha;
+                                v.z = __uint_as_float(r[j + 2]) * alpha;
+                                v.w = __uint_as_float(r[j + 3]) * alpha;
+                                *reinterpret_cast<float4 *>(yrow + j) = v;
+                                fsum = fmaf(v.x, v.x, fsum);
+                                fsum = fmaf(v.y, v.y, fsum);
+                                fsum = fmaf(v.z, v.z, fsum);
+                                fsum = fmaf(v.w, v.w, fsum);
+                            } else {
+                                const float4 y = *reinterpret_cast<const float4 *>(yrow + j);
+                                float4 cs = make_float4(1.f, 1.f, 1.f, 1.f);
+                                if (p.col_scale) cs = __ldg(reinterpret_cast<const float4 *>(p.col_scale + col0 + j));
+                                const float d0 = y.x - __uint_as_float(r[j]) * (alpha * cs.x);
+                                const float d1 = y.y - __uint_as_float(r[j + 1]) * (alpha * cs.y);
+                                const float d2 = y.z - __uint_as_float(r[j + 2]) * (alpha * cs.z);
+                                const float d3 = y.w - __uint_as_float(r[j + 3]) * (alpha * cs.w);
+                                fsum = fmaf(d0, d0, fsum);
+                                fsum = fmaf(d1, d1, fsum);
+                                fsum = fmaf(d2, d2, fsum);
+                                fsum = fmaf(d3, d3, fsum);
+                            }
+                        }
+                    } else {
+                        for (int j = 0; j < 32 && col0 + j < p.N; ++j) {  // ragged right edge
+                            const float a = __uint_as_float(r[j]);
+                            if (p.mode == 0) {
+                                const float v = a * alpha;
+                                yrow[j] = v;
+                                fsum = fmaf(v, v, fsum);
+                            } else {
+                                const float cs = p.col_scale ? p.col_scale[col0 + j] : 1.0f;
+                                const float d = yrow[j] - a * (alpha * cs);
+                                fsum = fmaf(d, d, fsum);
+                            }
+                        }
+                    }
+                }
+            }
+            dsum += (double)fsum;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty_bar[buf]);
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        if (lane == 0) red[q] = dsum;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        p.partials[blockIdx.x] = (red[0] + red[1]) + (red[2] + red[3]);
+        if (err) atomicOr(p.status, MOFQ_STATUS_TIMEOUT);
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+#undef err
+}
+
+// ---- helper kernels -------------------------------------------------------------------------------------------
+// bf16 activations -> fp16 operand: scaled by the power of two that puts the tensor's abs-max in [2^13, 2^14), which
+// keeps every bf16 value exact in fp16 unless it is more than 2^27 times smaller than the abs-max.
+__global__ void __launch_bounds__(256)
+x_bf16_to_f16(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, const WsHeader *hdr, uint16_t *out, float *alpha_out)
+{
+    const uint32_t m16 = hdr->absmax_bits;
+    const int e = (int)(m16 >> 7) - 127;  // bf16 exponent of the abs-max (0 -> treated as tiny)
+    const int pw = m16 ? 13 - e : 0;
+    const float mult = exp2f((float)max(min(pw, 126), -126));
+    if (blockIdx.x == 0 && threadIdx.x == 0) *alpha_out = exp2f((float)-max(min(pw, 126), -126));
+    const int cpr = cols >> 3;
+    const long long total = rows * cpr;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / cpr;
+        const int c = (int)(i - r * cpr);
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float lo = __uint_as_float(w[k] << 16) * mult, hi = __uint_as_float(w[k] & 0xFFFF0000u) * mult;
+            o[k] = (uint32_t)__half_as_ushort(__float2half_rn(lo)) | ((uint32_t)__half_as_ushort(__float2half_rn(hi)) << 16);
+        }
+        *reinterpret_cast<uint4 *>(out + r * cols + (long long)c * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+__global__ void set_scalar(float *p, float v) { *p = v; }
+
+struct LayerFinalize {
+    const double *partials;  // [(1 + n_cand)][stride]
+    int stride, n_ctas, n_cand;
+    double inv_n;
+    mofq_result *res;
+    float *mse_out, *nsr_out;
+    int32_t *status;         // device status word: cleared after it is read when a record is written
+};
+
+__global__ void __launch_bounds__(32)
+layer_finalize(const LayerFinalize f)
+{
+    double tot[1 + MOFQ_MAX_CAND];
+    for (int k = 0; k <= f.n_cand; ++k) {
+        double s = 0.0;
+        for (int c = threadIdx.x; c < f.n_ctas; c += 32) s += f.partials[(size_t)k * f.stride + c];
+#pragma unroll
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        tot[k] = s;
+    }
+    if (threadIdx.x != 0) return;
+    double best = INFINITY, second = INFINITY;
+    int chosen = -1;
+    mofq_result r;
+    for (int i = 0; i < MOFQ_MAX_CAND; ++i) r.error[i] = r.nsr[i] = 0.0f;
+    for (int i = 0; i < f.n_cand; ++i) {
+        const double mse = tot[1 + i] * f.inv_n, nsr = tot[0] > 0.0 ? tot[1 + i] / tot[0] : 0.0;
+        r.error[i] = (float)mse;
+        r.nsr[i] = (float)nsr;
+        if (f.mse_out) f.mse_out[i] = (float)mse;
+        if (f.nsr_out) f.nsr_out[i] = (float)nsr;
+        // Algorithm 1: strict '<' in the caller's candidate order
+        if (mse < best) {
+            second = best;
+            best = mse;
+            chosen = i;
+        } else if (mse < second) {
+            second = mse;
+        }
+    }
+    if (f.res) {
+        r.chosen = chosen;
+        r.status = atomicExch(f.status, 0);
+        r.rel_margin = best > 0.0 ? (float)((second - best) / best) : INFINITY;
+        r.reserved = 0;
+        *f.res = r;
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [rows, cols] 16-bit row-major tensor with leading dimension ld -> map with a {BK, box_rows} box and the 128-byte swizzle
+int make_map(CUtensorMap *map, const void *base, int dtype, long long rows, long long cols, long long ld, int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled();
+    if (!fn) return MOFQ_ERR_CUDA;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult rc = fn(map, dtype == MOFQ_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                           const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS ? MOFQ_OK : MOFQ_ERR_CUDA;
+}
+
+size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// Workspace of the layer metric, after the scoring workspace:
+struct LayerWs {
+    size_t x16, cx, cw, y, sw, scal, partials, total;
+};
+LayerWs layer_ws_layout(long long T, long long n_in, long long n_out)
+{
+    LayerWs w{};
+    size_t off = 0;
+    w.x16 = off; off += align256((size_t)T * n_in * 2);
+    w.cx = off;  off += align256((size_t)T * n_in * 2);
+    w.cw = off;  off += align256((size_t)n_out * n_in * 2);
+    w.y = off;   off += align256((size_t)T * n_out * 4);
+    w.sw = off;  off += align256((size_t)n_out * 4);
+    w.scal = off; off += 256;  // [0] reference alpha, [1] activation scale of the current format
+    w.partials = off; off += align256(sizeof(double) * (1 + MOFQ_MAX_CAND) * kMaxGemmCtas);
+    w.total = off;
+    return w;
+}
+
+int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, long long b_rows, long long b_ld, long long K,
+             int dtype, int mode, float *Y, const float *alpha, const float *col_scale, double *partials, int32_t *status,
+             int *grid_out, cudaStream_t st)
+{
+    CUtensorMap map_a, map_b;
+    if (int rc = make_map(&map_a, a, dtype, a_rows, K, a_ld, BM)) return rc;
+    if (int rc = make_map(&map_b, b, dtype, b_rows, K, b_ld, BN)) return rc;
+    GemmParams p{};
+    p.M = (int)a_rows;
+    p.N = (int)b_rows;
+    p.K = (int)K;
+    p.mode = mode;
+    p.Y = Y;
+    p.alpha = alpha;
+    p.col_scale = col_scale;
+    p.partials = partials;
+    p.status = status;
+    const uint32_t fmt = dtype == MOFQ_F16 ? 0u : 1u;
+    p.idesc = (1u << 4) /* fp32 accumulator */ | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    const int tiles = (int)(((a_rows + BM - 1) / BM) * ((b_rows + BN - 1) / BN));
+    const int grid = std::min(tiles, std::min(sm_count(), kMaxGemmCtas));
+    const size_t smem = (size_t)kStages * kStageBytes + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(gemm_err_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MOFQ_ERR_CUDA;
+        }
+        attr_set = true;
+    }
+    gemm_err_kernel<<<grid, kGemmThreads, smem, st>>>(map_a, map_b, p);
+    if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+    *grid_out = grid;
+    return MOFQ_OK;
+}
+
+}  // namespace
+
+size_t layer_metric_ws_bytes(const mofq_layer *layers, int n_layers, const mofq_config *)
+{
+    size_t need = 0;
+    for (int i = 0; i < n_layers; ++i)
+        need = std::max(need, layer_ws_layout(layers[i].X.rows, layers[i].W.cols, layers[i].W.rows).total);
+    return need;
+}
+
+int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *res, float *mse_out, float *nsr_out,
+                     void *workspace, size_t workspace_bytes, cudaStream_t st)
+{
+    const mofq_tensor &W = L.W, &X = L.X;
+    if (X.cols != W.cols) return MOFQ_ERR_INVALID_ARG;
+    if (cfg->w_gran != MOFQ_PER_CHANNEL) return MOFQ_ERR_UNSUPPORTED;               // scales must factor out of the contraction
+    if (!cfg->is_w_only && cfg->a_gran != MOFQ_PER_TENSOR) return MOFQ_ERR_UNSUPPORTED;
+    if (X.dtype == MOFQ_F16 && W.dtype == MOFQ_BF16) return MOFQ_ERR_UNSUPPORTED;    // no exact common 16-bit operand type
+    if (W.rows > 0x7fffffffLL || X.rows > 0x7fffffffLL || W.cols > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+    FmtDesc fd[MOFQ_MAX_CAND];
+    for (int i = 0; i < cfg->n_candidates; ++i) {
+        if (!describe_format(cfg->candidates[i], &fd[i])) return MOFQ_ERR_INVALID_ARG;
+        if (fd[i].bits != cfg->bit_width) return MOFQ_ERR_UNSUPPORTED;
+    }
+    const long long T = X.rows, n_in = W.cols, n_out = W.rows;
+    const LayerWs lw = layer_ws_layout(T, n_in, n_out);
+    const size_t base_off = align256(score_ws_bytes());
+    if (workspace_bytes < base_off + lw.total) return MOFQ_ERR_WORKSPACE_TOO_SMALL;
+    char *base = static_cast<char *>(workspace) + base_off;
+    WsHeader *hdr = static_cast<WsHeader *>(workspace);
+    uint16_t *x16 = reinterpret_cast<uint16_t *>(base + lw.x16), *cx = reinterpret_cast<uint16_t *>(base + lw.cx);
+    uint16_t *cw = reinterpret_cast<uint16_t *>(base + lw.cw);
+    float *Y = reinterpret_cast<float *>(base + lw.y), *sw = reinterpret_cast<float *>(base + lw.sw);
+    float *scal = reinterpret_cast<float *>(base + lw.scal);
+    double *partials = reinterpret_cast<double *>(base + lw.partials);
+    const int op_dtype = W.dtype;  // operand type of every GEMM of this layer
+
+    // reference operand for X (and its abs-max, which also serves the per-tensor activation scale)
+    const void *xa = X.data;
+    long long xa_ld = X.ld;
+    if (X.dtype != op_dtype) {  // bf16 activations with fp16 weights
+        if (cudaMemsetAsync(&hdr->absmax_bits, 0, sizeof(uint32_t), st) != cudaSuccess) return MOFQ_ERR_CUDA;
+        if (int rc = launch_absmax(X, hdr, st)) return rc;
+        const long long total = T * (n_in / 8);
+        const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
+        x_bf16_to_f16<<<grid, 256, 0, st>>>(static_cast<const uint16_t *>(X.data), T, (int)n_in, X.ld, hdr, x16, scal);
+        if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+        xa = x16;
+        xa_ld = n_in;
+    } else {
+        set_scalar<<<1, 1, 0, st>>>(scal, 1.0f);
+        if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+    }
+    int grid_used = 0, max_grid = 0;
+    if (int rc = run_gemm(xa, T, xa_ld, W.data, n_out, W.ld, n_in, op_dtype, 0, Y, scal, nullptr, partials, &hdr->status, &grid_used, st))
+        return rc;
+    max_grid = grid_used;
+    for (int i = 0; i < cfg->n_candidates; ++i) {  // Algorithm 1: for format in format_candidates
+        if (int rc = launch_emit(W, fd[i], MOFQ_PER_CHANNEL, 0, nullptr, nullptr, sw, nullptr, cw, op_dtype, hdr, st)) return rc;
+        const void *a = xa;
+        long long a_ld = xa_ld;
+        const float *alpha = scal;
+        if (!cfg->is_w_only) {
+            if (int rc = launch_emit(X, fd[i], MOFQ_PER_TENSOR, 0, nullptr, nullptr, scal + 1, nullptr, cx, op_dtype, hdr, st)) return rc;
+            a = cx;
+            a_ld = n_in;
+            alpha = scal + 1;
+        }
+        if (int rc = run_gemm(a, T, a_ld, cw, n_out, n_in, n_in, op_dtype, 1, Y, alpha, sw, partials + (size_t)(1 + i) * kMaxGemmCtas,
+                              &hdr->status, &grid_used, st))
+            return rc;
+        max_grid = std::max(max_grid, grid_used);
+    }
+    LayerFinalize f{};
+    f.partials = partials;
+    f.stride = kMaxGemmCtas;
+    f.n_ctas = max_grid;
+    f.n_cand = cfg->n_candidates;
+    f.inv_n = 1.0 / ((double)T * (double)n_out);
+    f.res = res;
+    f.mse_out = mse_out;
+    f.nsr_out = nsr_out;
+    f.status = &hdr->status;
+    layer_finalize<<<1, 32, 0, st>>>(f);
+    if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+    return MOFQ_OK;
 }
 
 }  // namespace mofq
