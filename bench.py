@@ -112,6 +112,25 @@ def cpu_oracle_sample(workload, budget_s=12.0, max_chunks=64):
     grans = [{"channel": orc.PER_CHANNEL, "group": orc.PER_GROUP, "tensor": orc.PER_TENSOR}[g] for g in wl["w_gran"]]
     orc.lib()
     done_bytes, t_total, chunks = 0, 0.0, 0
+    if wl["metric"] == "layer_output":
+        # the double-precision triple loop is far too slow for a whole layer: score 256 output rows against 64 of the
+        # calibration tokens and scale the throughput by 64 / tokens (the oracle's cost is linear in the token count)
+        t_s, rows = 64, 256
+        while t_total < budget_s and chunks < max_chunks:
+            li = chunks % len(layers)
+            name, out_f, in_f = layers[li]
+            w = inputs.weight_cpu(wl["w_kind"], min(rows, out_f), in_f, wl["seed"], li, **wl["w_args"])
+            x = inputs.activation_cpu(t_s, in_f, wl["seed"], li, **wl["a_args"])
+            t0 = time.perf_counter()
+            errs = [orc.layer_output_error(x, w, f, False)[0] for f in cands]
+            orc.select(errs)
+            t_total += time.perf_counter() - t0
+            done_bytes += w.numel() * 2
+            chunks += 1
+        scale = t_s / wl["tokens"]
+        return {"value": done_bytes / t_total / 1e9 * scale, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+                "sample": f"{chunks} slices of {rows} output rows x {t_s} tokens from the first layers, {t_total:.1f} s of CPU "
+                          f"work, layer-output criterion; value extrapolated to {wl['tokens']} tokens (x{scale:.4f})"}, done_bytes * scale, t_total
     while t_total < budget_s and chunks < max_chunks:
         name, out_f, in_f = layers[chunks % len(layers)]
         rows = min(out_f, 1024)
@@ -180,28 +199,69 @@ def main():
     mofq.lib()
 
     wl = inputs.WORKLOADS[args.workload]
-    if wl["metric"] != "tensor":
-        raise SystemExit("this bench times the tensor-MSE workloads; the layer-output criterion is not built yet")
+    layer_metric = wl["metric"] == "layer_output"
     shapes = inputs.workload_layers(args.workload, args.blocks)
     # weak scaling: every rank scores a whole model of its own (seed offset by rank); no data-path collective
     seed = wl["seed"] + 1000 * rank
-    layers = []
-    for li, (_, out_f, in_f) in enumerate(shapes):
-        w = torch.empty((out_f, in_f), dtype=torch.float16, device=dev)
-        inputs.device_weight(w, wl["w_kind"], seed, li, **wl["w_args"])
-        layers.append(w)
-    n_elems = sum(w.numel() for w in layers)
+    n_elems = sum(o * i for _, o, i in shapes)
     fp16_bytes = 2 * n_elems
+    T = wl["tokens"]
     grans = wl["w_gran"]
-    cfg = mofq.make_config(wl["bits"], wl["candidates"], metric="tensor", w_gran=grans[0], w_group=wl["group"],
-                           w_gran2=grans[1] if len(grans) > 1 else None)
-    n_rec = len(layers) * len(grans)
+    cfg = mofq.make_config(wl["bits"], wl["candidates"], metric=wl["metric"], is_w_only=not layer_metric,
+                           w_gran=grans[0], w_group=wl["group"], w_gran2=grans[1] if len(grans) > 1 else None)
+    n_rec = len(shapes) * len(grans)
     results = torch.empty(n_rec * B.RESULT_BYTES, dtype=torch.uint8, device=dev)
-    prepared = mofq.prepare_layers(layers)          # marshal the layer list once; a step is one C-ABI call
-    ws = torch.empty(mofq.workspace_bytes(prepared, cfg), dtype=torch.uint8, device=dev)
+    x_bytes = sum(2 * T * i for _, o, i in shapes) if layer_metric else 0
+    streaming = fp16_bytes + x_bytes > 100e9          # synthesise each layer on the device inside the step
+    layers = []
+    if not streaming:
+        for li, (_, out_f, in_f) in enumerate(shapes):
+            w = torch.empty((out_f, in_f), dtype=torch.float16, device=dev)
+            inputs.device_weight(w, wl["w_kind"], seed, li, **wl["w_args"])
+            if layer_metric:
+                x = torch.empty((T, in_f), dtype=torch.bfloat16, device=dev)
+                inputs.device_activation(x, seed, li, **wl["a_args"])
+                layers.append((w, x))
+            else:
+                layers.append(w)
+        prepared = mofq.prepare_layers(layers)          # marshal the layer list once; a step is one C-ABI call
+        ws = torch.empty(mofq.workspace_bytes(prepared, cfg), dtype=torch.uint8, device=dev)
 
-    def step():
-        mofq.select_formats(prepared, cfg, workspace=ws, results=results, parse=False)
+        def step():
+            mofq.select_formats(prepared, cfg, workspace=ws, results=results, parse=False)
+
+        synth_ms = 0.0
+    else:
+        max_w = max(o * i for _, o, i in shapes)
+        max_x = max(T * i for _, o, i in shapes)
+        wbuf = torch.empty(max_w, dtype=torch.float16, device=dev)
+        xbuf = torch.empty(max_x, dtype=torch.bfloat16, device=dev)
+        views = [(wbuf[:o * i].view(o, i), xbuf[:T * i].view(T, i)) for _, o, i in shapes]
+        big = max(views, key=lambda v: v[0].numel())
+        ws = torch.empty(mofq.workspace_bytes([big], cfg), dtype=torch.uint8, device=dev)
+        preps = [mofq.prepare_layers([v]) for v in views]
+        res_views = [results[li * B.RESULT_BYTES:(li + 1) * B.RESULT_BYTES] for li in range(len(shapes))]
+
+        def synth(li):
+            w, x = views[li]
+            inputs.device_weight(w, wl["w_kind"], seed, li, **wl["w_args"])
+            inputs.device_activation(x, seed, li, **wl["a_args"])
+
+        def step():
+            for li in range(len(shapes)):                # one layer resident at a time (stream-ordered reuse of the buffers)
+                synth(li)
+                mofq.select_formats(preps[li], cfg, workspace=ws, results=res_views[li], parse=False)
+
+        torch.cuda.synchronize()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for li in range(len(shapes)):
+            synth(li)
+        s0.record()
+        for li in range(len(shapes)):
+            synth(li)
+        s1.record()
+        torch.cuda.synchronize()
+        synth_ms = s0.elapsed_time(s1)
 
     def barrier():
         if world > 1:
@@ -238,7 +298,7 @@ def main():
 
     # end to end through the host-buffer entry point (N ranks each copy their own model)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not streaming and not layer_metric:
         host_layers = [torch.empty(w.shape, dtype=w.dtype, pin_memory=True) for w in layers]
         for h, w in zip(host_layers, layers):
             h.copy_(w)
@@ -270,7 +330,9 @@ def main():
         peaks, which = measured_peaks()
         peak = float(peaks["hbm_gbs"])
         # algorithmic bytes: 2 B per element read once (+ 4 B per 128 elements of scale state never leaves the SM)
-        launches_per_step = len(layers)
+        F = cfg.n_candidates
+        flops = sum(2.0 * T * o * i * (1 + F) for _, o, i in shapes) if layer_metric else 0.0
+        launches_per_step = len(shapes) * (3 + 4 * F + 2) if layer_metric else (3 + (len(shapes) + 63) // 64 if grans == ("group",) else len(shapes))
         roofline = {"bound": "hbm", "kernel": "kq_score_*", "achieved": fp16_bytes / (ms_per_step * 1e-3) / 1e9,
                     "peak": peak, "peak_source": f"of {which}", "unit": "GB/s",
                     "frac": fp16_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
@@ -281,12 +343,21 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "layers": len(layers), "elements": n_elems, "fp16_GB": fp16_bytes / 1e9,
+            "config": {"workload": args.workload, "layers": len(shapes), "elements": n_elems, "fp16_GB": fp16_bytes / 1e9,
                        "candidates": list(wl["candidates"]), "granularity": list(grans), "group": wl["group"],
-                       "criterion": "tensor_mse", "l2": "inputs larger than L2" if fp16_bytes > 2.5e8 else "inputs fit in L2",
+                       "criterion": wl["metric"], "tokens": T, "streaming_synthesis": streaming, "synthesis_ms_per_step": synth_ms,
+                       "l2": "inputs larger than L2" if fp16_bytes > 2.5e8 else "inputs fit in L2",
                        "model_select_time_ms": ms_per_step, "fp_share": fp_share, "min_rel_margin": min_margin},
             "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * launches_per_step, "roofline": roofline,
         }
+        if layer_metric:
+            gemm_ms = ms_per_step - synth_ms
+            tf = flops / (gemm_ms * 1e-3) / 1e12
+            tpeak = float(peaks.get("bf16_tflops_sustained", 1400.0))
+            out["roofline"] = {"bound": "tensor", "kernel": "gemm_err_kernel", "achieved": tf, "peak": tpeak,
+                               "peak_source": f"of {which} (sustained 16-bit dense; fp16 operands share the bf16 rate)",
+                               "unit": "TFLOP/s", "frac": tf / tpeak, "flops_per_step": flops,
+                               "note": "whole step minus synthesis time; includes the operand-preparation kernels", "traffic": None}
         if not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_oracle_sample(args.workload)[0]
         print(json.dumps(out))

@@ -26,12 +26,19 @@
 namespace mofq {
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64;
-constexpr int kStages = 6;
-constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2;
-constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int BM = 128;
+constexpr int kRowBytes = 128;  // bytes of K per tile row: 64 16-bit or 128 8-bit elements (one 128-byte swizzle row)
+constexpr int kABytes = BM * kRowBytes;
+constexpr int kRingBytes = 192 * 1024;
 constexpr int kGemmThreads = 192;  // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-5: epilogue
-constexpr int kTmemCols = 256;     // two accumulators of BN columns
+// Tile width BN is 128 or 256: the wider tile moves 25% fewer operand bytes per flop (the main loop is bound by
+// L2 -> shared-memory traffic), the narrower one quantises better onto 148 SMs.  Two accumulators of BN columns.
+template <int BN> struct TileCfg {
+    static constexpr int kBBytes = BN * kRowBytes;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kStages = kRingBytes / kStageBytes;  // 6 (BN=128) or 4 (BN=256)
+    static constexpr int kTmemCols = 2 * BN;
+};
 constexpr long long kWaitCycles = 4000000000LL;
 constexpr int kMaxGemmCtas = 148 * 2;
 
@@ -78,6 +85,16 @@ __device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t a_desc, uin
     asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p; }"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p; }"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 // 32 lanes x 32 consecutive fp32 columns: thread i receives row (lane base + i)
 __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -110,11 +127,16 @@ struct GemmParams {
     double *partials;         // one double per CTA
     int32_t *status;          // device status word (timeout)
     uint32_t idesc;
+    int kind;                 // operand kind of the MMA: KIND_F16 (fp16/bf16), KIND_I8 (int8 -> int32), KIND_F8 (e4m3/e5m2)
+    int bk;                   // elements of K per tile row (64 or 128)
 };
+enum { KIND_F16 = 0, KIND_I8 = 1, KIND_F8 = 2 };
 
+template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
 {
+    constexpr int kStages = TileCfg<BN>::kStages, kStageBytes = TileCfg<BN>::kStageBytes, kTmemCols = TileCfg<BN>::kTmemCols;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], tfull_bar[2], tempty_bar[2];
     __shared__ uint32_t tmem_base_slot;
@@ -127,7 +149,7 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
     const int n_tiles = tiles_m * tiles_n;
-    const int kblocks = (p.K + BK - 1) / BK;
+    const int kblocks = (p.K + p.bk - 1) / p.bk;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -156,14 +178,14 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (lane == 0) {
             int it = 0;
             for (int tile = blockIdx.x; tile < n_tiles && !err; tile += gridDim.x) {
-                const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+                const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;  // m fastest: co-running tiles share a B tile
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % kStages;
                     if (!mbar_wait(&empty_bar[s], ((it / kStages) & 1) ^ 1, perr)) break;
                     mbar_expect_tx(&full_bar[s], kStageBytes);
                     unsigned char *st = smem + (size_t)s * kStageBytes;
-                    tma_load_2d(st, &map_a, kb * BK, m0, &full_bar[s]);
-                    tma_load_2d(st + kABytes, &map_b, kb * BK, n0, &full_bar[s]);
+                    tma_load_2d(st, &map_a, kb * p.bk, m0, &full_bar[s]);
+                    tma_load_2d(st + kABytes, &map_b, kb * p.bk, n0, &full_bar[s]);
                 }
             }
             if (err) {  // let copies that are still in flight land before the shared memory is given back
@@ -190,8 +212,12 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
                     const uint64_t a_desc = smem_desc_k_major_sw128(sa), b_desc = smem_desc_k_major_sw128(sa + kABytes);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)  // each step advances 16 elements = 32 bytes inside the swizzled row
-                        tc_mma_f16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc, (kb | k) != 0);
+                    for (int k = 0; k < kRowBytes / 32; ++k) {  // one MMA consumes 32 bytes of K (16 x 16-bit or 32 x 8-bit)
+                        const uint64_t ad = a_desc + (uint64_t)(2 * k), bd = b_desc + (uint64_t)(2 * k);
+                        if (p.kind == KIND_F16) tc_mma_f16(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                        else if (p.kind == KIND_I8) tc_mma_i8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                        else tc_mma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                    }
                     tc_commit(&empty_bar[s]);  // the stage is free once these MMAs have read it
                 }
                 if (!ok) break;
@@ -206,7 +232,7 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         int local = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++local) {
             const int buf = local & 1;
-            const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+            const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;  // m fastest: co-running tiles share a B tile
             if (!mbar_wait(&tfull_bar[buf], (local >> 1) & 1, perr)) break;
             tc_fence_after();
             const int row = m0 + q * 32 + lane;
@@ -216,6 +242,10 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 uint32_t r[32];
                 tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), r);
                 const int col0 = n0 + c * 32;
+                if (p.kind == KIND_I8) {  // exact integer dot products -> float
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint((float)(int)r[j]);
+                }
                 if (row < p.M) {
                     float *yrow = p.Y + (size_t)row * p.N + col0;
                     if (col0 + 32 <= p.N && (p.N & 3) == 0) {
@@ -384,15 +414,20 @@ EncodeTiledFn encode_tiled()
 }
 
 // [rows, cols] 16-bit row-major tensor with leading dimension ld -> map with a {BK, box_rows} box and the 128-byte swizzle
-int make_map(CUtensorMap *map, const void *base, int dtype, long long rows, long long cols, long long ld, int box_rows)
+// elem: MOFQ_F16, MOFQ_BF16 or kElemU8
+constexpr int kElemU8 = 2;
+int make_map(CUtensorMap *map, const void *base, int elem, long long rows, long long cols, long long ld, int box_rows)
 {
     EncodeTiledFn fn = encode_tiled();
     if (!fn) return MOFQ_ERR_CUDA;
+    const int esize = elem == kElemU8 ? 1 : 2;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * esize};
+    const cuuint32_t box[2] = {(cuuint32_t)(kRowBytes / esize), (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult rc = fn(map, dtype == MOFQ_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+    const CUtensorMapDataType dt = elem == kElemU8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                   : elem == MOFQ_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUresult rc = fn(map, dt, 2,
                            const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return rc == CUDA_SUCCESS ? MOFQ_OK : MOFQ_ERR_CUDA;
@@ -419,13 +454,22 @@ LayerWs layer_ws_layout(long long T, long long n_in, long long n_out)
     return w;
 }
 
+// op: MOFQ_F16 / MOFQ_BF16 (16-bit operands), or an 8-bit mofq_format (MOFQ_INT8, MOFQ_FP8_E4M3, MOFQ_FP8_E5M2) + 100
+constexpr int kOp8 = 100;
 int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, long long b_rows, long long b_ld, long long K,
-             int dtype, int mode, float *Y, const float *alpha, const float *col_scale, double *partials, int32_t *status,
+             int op, int mode, float *Y, const float *alpha, const float *col_scale, double *partials, int32_t *status,
              int *grid_out, cudaStream_t st)
 {
+    // tile width: waves x relative tile cost (operand bytes per tile: 32 KB vs 48 KB per k-block)
+    const int nsm = sm_count();
+    const long long mt = (a_rows + BM - 1) / BM;
+    const long long t128 = mt * ((b_rows + 127) / 128), t256 = mt * ((b_rows + 255) / 256);
+    const double c128 = (double)((t128 + nsm - 1) / nsm) * 1.0, c256 = (double)((t256 + nsm - 1) / nsm) * 1.5;
+    const int bn = c256 < c128 ? 256 : 128;
     CUtensorMap map_a, map_b;
-    if (int rc = make_map(&map_a, a, dtype, a_rows, K, a_ld, BM)) return rc;
-    if (int rc = make_map(&map_b, b, dtype, b_rows, K, b_ld, BN)) return rc;
+    const int elem = op >= kOp8 ? kElemU8 : op;
+    if (int rc = make_map(&map_a, a, elem, a_rows, K, a_ld, BM)) return rc;
+    if (int rc = make_map(&map_b, b, elem, b_rows, K, b_ld, bn)) return rc;
     GemmParams p{};
     p.M = (int)a_rows;
     p.N = (int)b_rows;
@@ -436,21 +480,29 @@ int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, lon
     p.col_scale = col_scale;
     p.partials = partials;
     p.status = status;
-    const uint32_t fmt = dtype == MOFQ_F16 ? 0u : 1u;
-    p.idesc = (1u << 4) /* fp32 accumulator */ | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-    const int tiles = (int)(((a_rows + BM - 1) / BM) * ((b_rows + BN - 1) / BN));
+    // instruction descriptor: accumulator type [4,6), A type [7,10), B type [10,13), both K-major, N/8 at [17,23), M/16 at [24,29)
+    uint32_t cfmt, abfmt;
+    if (op == kOp8 + MOFQ_INT8) {
+        p.kind = KIND_I8; cfmt = 2u /* s32 */; abfmt = 1u /* signed 8-bit */;
+    } else if (op >= kOp8) {
+        p.kind = KIND_F8; cfmt = 1u /* f32 */; abfmt = op == kOp8 + MOFQ_FP8_E4M3 ? 0u : 1u /* e4m3 : e5m2 */;
+    } else {
+        p.kind = KIND_F16; cfmt = 1u; abfmt = op == MOFQ_F16 ? 0u : 1u /* f16 : bf16 */;
+    }
+    p.bk = op >= kOp8 ? kRowBytes : kRowBytes / 2;
+    p.idesc = (cfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    const int tiles = (int)(((a_rows + BM - 1) / BM) * ((b_rows + bn - 1) / bn));
     const int grid = std::min(tiles, std::min(sm_count(), kMaxGemmCtas));
-    const size_t smem = (size_t)kStages * kStageBytes + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_err_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    const size_t smem = (size_t)kRingBytes + 1024;
+    auto launch = [&](auto kernel) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
             (void)cudaGetLastError();
             return MOFQ_ERR_CUDA;
         }
-        attr_set = true;
-    }
-    gemm_err_kernel<<<grid, kGemmThreads, smem, st>>>(map_a, map_b, p);
-    if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+        kernel<<<grid, kGemmThreads, smem, st>>>(map_a, map_b, p);
+        return cudaGetLastError() == cudaSuccess ? MOFQ_OK : MOFQ_ERR_CUDA;
+    };
+    if (int rc = bn == 256 ? launch(gemm_err_kernel<256>) : launch(gemm_err_kernel<128>)) return rc;
     *grid_out = grid;
     return MOFQ_OK;
 }
@@ -508,22 +560,29 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
         set_scalar<<<1, 1, 0, st>>>(scal, 1.0f);
         if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
     }
+    // WA with 8-bit candidates: the codes themselves are the tensor-core operands (int8 / e4m3 / e5m2 kinds)
+    const bool native8 = !cfg->is_w_only && cfg->bit_width == 8 && (n_in % 16) == 0;
     int grid_used = 0, max_grid = 0;
     if (int rc = run_gemm(xa, T, xa_ld, W.data, n_out, W.ld, n_in, op_dtype, 0, Y, scal, nullptr, partials, &hdr->status, &grid_used, st))
         return rc;
     max_grid = grid_used;
     for (int i = 0; i < cfg->n_candidates; ++i) {  // Algorithm 1: for format in format_candidates
-        if (int rc = launch_emit(W, fd[i], MOFQ_PER_CHANNEL, 0, nullptr, nullptr, sw, nullptr, cw, op_dtype, hdr, st)) return rc;
+        if (int rc = launch_emit(W, fd[i], MOFQ_PER_CHANNEL, 0, nullptr, native8 ? cw : nullptr, sw, nullptr, native8 ? nullptr : cw,
+                                 op_dtype, hdr, st))
+            return rc;
         const void *a = xa;
         long long a_ld = xa_ld;
         const float *alpha = scal;
         if (!cfg->is_w_only) {
-            if (int rc = launch_emit(X, fd[i], MOFQ_PER_TENSOR, 0, nullptr, nullptr, scal + 1, nullptr, cx, op_dtype, hdr, st)) return rc;
+            if (int rc = launch_emit(X, fd[i], MOFQ_PER_TENSOR, 0, nullptr, native8 ? cx : nullptr, scal + 1, nullptr,
+                                     native8 ? nullptr : cx, op_dtype, hdr, st))
+                return rc;
             a = cx;
             a_ld = n_in;
             alpha = scal + 1;
         }
-        if (int rc = run_gemm(a, T, a_ld, cw, n_out, n_in, n_in, op_dtype, 1, Y, alpha, sw, partials + (size_t)(1 + i) * kMaxGemmCtas,
+        const int op = native8 ? kOp8 + cfg->candidates[i] : op_dtype;
+        if (int rc = run_gemm(a, T, a_ld, cw, n_out, n_in, n_in, op, 1, Y, alpha, sw, partials + (size_t)(1 + i) * kMaxGemmCtas,
                               &hdr->status, &grid_used, st))
             return rc;
         max_grid = std::max(max_grid, grid_used);

@@ -52,6 +52,19 @@ def test_layer_output_error_matches_oracle(orc, dev, T, n_in, n_out, names, w_on
     assert rel_err(nsr.cpu().numpy(), want_nsr).max() < LAYER_RTOL, (nsr, want_nsr)
 
 
+def test_wide_tile_variant(orc, dev):
+    # 2 x 74 tiles of 128 x 256 fill 148 SMs in one wave, so the 256-wide tile is chosen; the right edge is ragged
+    T, n_in, n_out = 256, 128, 18936
+    w, x = _layer(dev, T, n_in, n_out, seed=55)
+    for names, w_only, bits in ((["INT8", "FP8_E4M3"], False, 8), (["INT4", "FP4_E2M1"], True, 4)):
+        cfg = mofq.make_config(bits, names, metric="layer_output", is_w_only=w_only)
+        mse, nsr, st = mofq.layer_output_error(x, w, cfg)
+        want_mse, want_nsr = _oracle(orc, w, x, names, w_only)
+        assert int(st.item()) == 0
+        assert rel_err(mse.cpu().numpy(), want_mse).max() < LAYER_RTOL
+        assert rel_err(nsr.cpu().numpy(), want_nsr).max() < LAYER_RTOL
+
+
 @pytest.mark.parametrize("xdtype,wdtype", [(torch.float16, torch.float16), (torch.bfloat16, torch.bfloat16)])
 def test_layer_output_error_dtype_combinations(orc, dev, xdtype, wdtype):
     w, x = _layer(dev, 256, 512, 256, seed=52, xdtype=xdtype, wdtype=wdtype, a_args=dict(ch_gain=8.0))
