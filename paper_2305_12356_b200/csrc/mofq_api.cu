@@ -211,7 +211,7 @@ int mofq_quantize_tensor(const mofq_tensor *x, int format, int gran, int group, 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
     return launch_emit(*x, f, gran, group, scales_in, codes_out, scales_out, dequant_out, nullptr, MOFQ_F16,
-                       static_cast<WsHeader *>(workspace), st);
+                       static_cast<WsHeader *>(workspace), st, format);
 }
 
 int mofq_tensor_error(const mofq_tensor *x, const int32_t *formats, int n, int gran, int gran2, int group,

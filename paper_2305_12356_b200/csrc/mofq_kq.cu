@@ -578,6 +578,110 @@ kq_emit(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, 
     if (status) atomicOr(&hdr->status, status);
 }
 
+// ---- fused code emission: per-channel scales, every requested format from ONE read of the row --------------------
+// Used for the tensor-core operands of the layer-output metric and for plain per-channel quantisation.
+// The FP codes come from the hardware converts (round-to-nearest-even, saturating, sign kept on zero), which
+// produce the same codes as the add/subtract rounding above; INT codes are the low bits of t + 1.5*2^23.
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("{ .reg .b16 t; cvt.rn.satfinite.e4m3x2.f32 t, %2, %1; cvt.u32.u16 %0, t; }" : "=r"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ uint32_t cvt_e5m2x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("{ .reg .b16 t; cvt.rn.satfinite.e5m2x2.f32 t, %2, %1; cvt.u32.u16 %0, t; }" : "=r"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("{ .reg .b8 t; .reg .b16 w; cvt.rn.satfinite.e2m1x2.f32 t, %2, %1; mov.b16 w, {t, 0}; cvt.u32.u16 %0, w; }" : "=r"(d) : "f"(lo), "f"(hi));
+    return d & 0xFFu;
+}
+
+// codes of 8 consecutive elements for one format, packed little-endian (8-bit: 64 bits, 4-bit: 32 bits)
+template <int DT>
+__device__ __forceinline__ uint64_t codes8(const uint4 v, int format, float inv)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint64_t out = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float lo, hi;
+        unpack2<DT>(w[i], lo, hi);
+        const float tl = __fmul_rn(lo, inv), th = __fmul_rn(hi, inv);
+        uint32_t c;  // two codes
+        int bits;
+        switch (format) {
+        case MOFQ_FP8_E4M3: c = cvt_e4m3x2(tl, th); bits = 8; break;
+        case MOFQ_FP8_E5M2: c = cvt_e5m2x2(tl, th); bits = 8; break;
+        case MOFQ_INT8:
+            c = (__float_as_uint(__fadd_rn(tl, kMagic)) & 0xFFu) | ((__float_as_uint(__fadd_rn(th, kMagic)) & 0xFFu) << 8);
+            bits = 8;
+            break;
+        case MOFQ_INT4:
+            c = (__float_as_uint(__fadd_rn(tl, kMagic)) & 0xFu) | ((__float_as_uint(__fadd_rn(th, kMagic)) & 0xFu) << 4);
+            bits = 4;
+            break;
+        default: c = cvt_e2m1x2(tl, th); bits = 4; break;  // both E2M1 variants: same spacing below the IEEE maximum 3
+        }
+        out |= (uint64_t)c << (i * 2 * bits);
+    }
+    return out;
+}
+
+struct EmitSet {
+    int n;
+    int format[3];
+    float Q[3];
+    unsigned char *codes[3];
+    float *scales[3];
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kRowThreads)
+kq_emit_codes_rows(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, EmitSet es, WsHeader *hdr)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ uint32_t mred[34];
+    __shared__ float inv_s[3];
+    const int chunks = cols >> 3;
+    const uint4 *row4 = reinterpret_cast<const uint4 *>(smem);
+    int status = 0;
+    for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(x + row * ld);
+        for (int q = threadIdx.x; q < chunks; q += kRowThreads) cp_async16(smem + q * 16, src + (size_t)q * 16);
+        cp_async_wait_all();
+        __syncthreads();
+        uint32_t m = 0;
+        for (int q = threadIdx.x; q < chunks; q += kRowThreads) m = absmax_chunk(row4[q], m);
+        const uint32_t m16 = block_max_u32(fold16(m), mred);
+        if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+        if ((int)threadIdx.x < es.n) {
+            float s, inv;
+            scale_pair(mag16_to_float<DT>(m16), es.Q[threadIdx.x], s, inv, status);
+            inv_s[threadIdx.x] = inv;
+            if (es.scales[threadIdx.x]) es.scales[threadIdx.x][row] = s;
+        }
+        __syncthreads();
+        for (int f = 0; f < es.n; ++f) {
+            const float inv = inv_s[f];
+            const int fmt = es.format[f];
+            const bool four = fmt == MOFQ_INT4 || fmt == MOFQ_FP4_E2M1 || fmt == MOFQ_FP4_E2M1_IEEE;
+            unsigned char *out = es.codes[f] + (four ? ((size_t)row * cols >> 1) : (size_t)row * cols);
+            for (int q = threadIdx.x; q < chunks; q += kRowThreads) {
+                const uint64_t c = codes8<DT>(row4[q], fmt, inv);
+                if (four) reinterpret_cast<uint32_t *>(out)[q] = (uint32_t)c;
+                else reinterpret_cast<uint2 *>(out)[q] = make_uint2((uint32_t)c, (uint32_t)(c >> 32));
+            }
+        }
+        __syncthreads();
+    }
+    if (status) atomicOr(&hdr->status, status);
+}
+
 // ---- host-side dispatch ----------------------------------------------------------------------------------
 #define MOFQ_CUDA_OK(expr)                      \
     do {                                        \
@@ -713,12 +817,48 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
     });
 }
 
+// Per-channel abs-max scales; codes (and scales) of n formats from one read.  formats[i] is a mofq_format.
+int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
+                           WsHeader *hdr, cudaStream_t st)
+{
+    if (n < 1 || n > 3 || x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)x.cols * 2;
+    if (smem > 200 * 1024) return MOFQ_ERR_UNSUPPORTED;
+    EmitSet es{};
+    es.n = n;
+    for (int i = 0; i < n; ++i) {
+        FmtDesc d;
+        if (!describe_format(formats[i], &d)) return MOFQ_ERR_INVALID_ARG;
+        es.format[i] = formats[i];
+        es.Q[i] = d.Q;
+        es.codes[i] = static_cast<unsigned char *>(codes[i]);
+        es.scales[i] = scales ? scales[i] : nullptr;
+    }
+    const uint16_t *xp = static_cast<const uint16_t *>(x.data);
+    auto launch = [&](auto kernel) {
+        if (int rc = set_smem(kernel, smem)) return rc;
+        const int occ = std::max(1, blocks_per_sm((const void *)kernel, kRowThreads, smem));
+        const int grid = (int)std::min<long long>(x.rows, (long long)sm_count() * occ);
+        kernel<<<grid, kRowThreads, smem, st>>>(xp, x.rows, (int)x.cols, x.ld, es, hdr);
+        MOFQ_CUDA_OK(cudaGetLastError());
+        return MOFQ_OK;
+    };
+    return x.dtype == MOFQ_F16 ? launch(kq_emit_codes_rows<0>) : launch(kq_emit_codes_rows<1>);
+}
+
 int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in, void *codes_out,
-                float *scales_out, void *dequant_out, void *values_out, int values_dtype, WsHeader *hdr, cudaStream_t st)
+                float *scales_out, void *dequant_out, void *values_out, int values_dtype, WsHeader *hdr, cudaStream_t st,
+                int format_id)
 {
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
     const int nsm = sm_count();
     if (x.cols > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+    if (gran == MOFQ_PER_CHANNEL && !scales_in && codes_out && !dequant_out && !values_out && x.cols * 2 <= 200 * 1024 &&
+        format_id >= 0) {
+        void *c[1] = {codes_out};
+        float *sc[1] = {scales_out};
+        return launch_emit_codes_rows(x, 1, &format_id, c, sc, hdr, st);
+    }
     if (gran == MOFQ_PER_TENSOR && !scales_in) {
         MOFQ_CUDA_OK(cudaMemsetAsync(&hdr->absmax_bits, 0, sizeof(uint32_t), st));
         const long long total = x.rows * (x.cols / 8);

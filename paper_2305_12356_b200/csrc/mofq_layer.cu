@@ -445,9 +445,9 @@ LayerWs layer_ws_layout(long long T, long long n_in, long long n_out)
     size_t off = 0;
     w.x16 = off; off += align256((size_t)T * n_in * 2);
     w.cx = off;  off += align256((size_t)T * n_in * 2);
-    w.cw = off;  off += align256((size_t)n_out * n_in * 2);
+    w.cw = off;  off += 3 * align256((size_t)n_out * n_in);   // 8-bit codes of up to 3 formats, or 16-bit values of one
     w.y = off;   off += align256((size_t)T * n_out * 4);
-    w.sw = off;  off += align256((size_t)n_out * 4);
+    w.sw = off;  off += 3 * align256((size_t)n_out * 4);
     w.scal = off; off += 256;  // [0] reference alpha, [1] activation scale of the current format
     w.partials = off; off += align256(sizeof(double) * (1 + MOFQ_MAX_CAND) * kMaxGemmCtas);
     w.total = off;
@@ -562,13 +562,32 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
     }
     // WA with 8-bit candidates: the codes themselves are the tensor-core operands (int8 / e4m3 / e5m2 kinds)
     const bool native8 = !cfg->is_w_only && cfg->bit_width == 8 && (n_in % 16) == 0;
+    // native path: the codes of every candidate from one read of W (one byte per element and format)
+    const bool fused_w = native8 && cfg->n_candidates <= 3;
+    const size_t cw_stride = align256((size_t)n_out * n_in), sw_stride = align256((size_t)n_out * 4) / 4;
+    if (fused_w) {
+        void *cptr[3];
+        float *sptr[3];
+        int fmts[3];
+        for (int i = 0; i < cfg->n_candidates; ++i) {
+            cptr[i] = reinterpret_cast<unsigned char *>(cw) + (size_t)i * cw_stride;
+            sptr[i] = sw + (size_t)i * sw_stride;
+            fmts[i] = cfg->candidates[i];
+        }
+        if (int rc = launch_emit_codes_rows(W, cfg->n_candidates, fmts, cptr, sptr, hdr, st)) return rc;
+    }
     int grid_used = 0, max_grid = 0;
     if (int rc = run_gemm(xa, T, xa_ld, W.data, n_out, W.ld, n_in, op_dtype, 0, Y, scal, nullptr, partials, &hdr->status, &grid_used, st))
         return rc;
     max_grid = grid_used;
     for (int i = 0; i < cfg->n_candidates; ++i) {  // Algorithm 1: for format in format_candidates
-        if (int rc = launch_emit(W, fd[i], MOFQ_PER_CHANNEL, 0, nullptr, native8 ? cw : nullptr, sw, nullptr, native8 ? nullptr : cw,
-                                 op_dtype, hdr, st))
+        const void *bw = cw;
+        const float *bsw = sw;
+        if (fused_w) {
+            bw = reinterpret_cast<unsigned char *>(cw) + (size_t)i * cw_stride;
+            bsw = sw + (size_t)i * sw_stride;
+        } else if (int rc = launch_emit(W, fd[i], MOFQ_PER_CHANNEL, 0, nullptr, native8 ? cw : nullptr, sw, nullptr,
+                                        native8 ? nullptr : cw, op_dtype, hdr, st))
             return rc;
         const void *a = xa;
         long long a_ld = xa_ld;
@@ -582,7 +601,7 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
             alpha = scal + 1;
         }
         const int op = native8 ? kOp8 + cfg->candidates[i] : op_dtype;
-        if (int rc = run_gemm(a, T, a_ld, cw, n_out, n_in, n_in, op, 1, Y, alpha, sw, partials + (size_t)(1 + i) * kMaxGemmCtas,
+        if (int rc = run_gemm(a, T, a_ld, bw, n_out, n_in, n_in, op, 1, Y, alpha, bsw, partials + (size_t)(1 + i) * kMaxGemmCtas,
                               &hdr->status, &grid_used, st))
             return rc;
         max_grid = std::max(max_grid, grid_used);
