@@ -28,6 +28,9 @@ if ROOT not in sys.path:
 
 METRIC = "GB/s of fp16 tensor quantized+scored (both formats)"
 UNIT = "GB/s"
+# DRAM bytes per element of kq_score_mt from the ncu capture summarised in profiles/ (read 809.54 MB + write 3.93 MB
+# for 404,750,336 elements on a 14-layer case; traffic is proportional to the elements processed)
+KQ_MT_DRAM_BYTES_PER_ELEMENT = (809.54e6 + 3.93e6) / 404750336
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
@@ -186,6 +189,7 @@ def main():
     import paper_2305_12356_b200 as mofq
     from paper_2305_12356_b200 import binding as B
     from paper_2305_12356_b200 import inputs
+    from paper_2305_12356_b200.sharded import max_over_ranks
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -282,11 +286,7 @@ def main():
     ev1.record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ev0.elapsed_time(ev1), dev)
     ms_per_step = ms / args.steps
     value = world * fp16_bytes / (ms_per_step * 1e-3) / 1e9
 
@@ -315,11 +315,7 @@ def main():
             hrecs = mofq.select_formats_host(host_layers, cfg, dev, workspace=hws)
         e1.record()
         barrier()
-        e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([e_ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = max_over_ranks(e0.elapsed_time(e1), dev)
         assert [r["chosen"] for r in hrecs] == [r["chosen"] for r in recs]
         e2e = {"value": world * fp16_bytes / (e_ms / args.e2e_steps * 1e-3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": fp16_bytes, "d2h_bytes_per_step": n_rec * B.RESULT_BYTES,
@@ -333,12 +329,15 @@ def main():
         F = cfg.n_candidates
         flops = sum(2.0 * T * o * i * (1 + F) for _, o, i in shapes) if layer_metric else 0.0
         launches_per_step = len(shapes) * (3 + 4 * F + 2) if layer_metric else (3 + (len(shapes) + 63) // 64 if grans == ("group",) else len(shapes))
-        roofline = {"bound": "hbm", "kernel": "kq_score_*", "achieved": fp16_bytes / (ms_per_step * 1e-3) / 1e9,
+        mt = grans == ("group",)
+        dom_launches = 1 if mt else len(shapes)      # launches of the dominant kernel per step
+        roofline = {"bound": "hbm", "kernel": "kq_score_mt" if mt else "kq_score_rows", "achieved": fp16_bytes / (ms_per_step * 1e-3) / 1e9,
                     "peak": peak, "peak_source": f"of {which}", "unit": "GB/s",
                     "frac": fp16_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
                     "frac_of_nominal_8TBs": fp16_bytes / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-                    "avg_launch_us": 1e3 * ms_per_step / launches_per_step,
-                    "algorithmic_bytes_per_launch": fp16_bytes / launches_per_step, "traffic": None}
+                    "launches_per_step": dom_launches, "avg_launch_us": 1e3 * ms_per_step / dom_launches,
+                    "algorithmic_bytes_per_launch": fp16_bytes / dom_launches,
+                    "traffic": KQ_MT_DRAM_BYTES_PER_ELEMENT * n_elems if mt else None}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
