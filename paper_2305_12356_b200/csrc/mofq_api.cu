@@ -116,7 +116,7 @@ int check_config(const mofq_config *cfg)
 
 // tensor metric for one layer: enqueue the scoring of W and the record(s) for it
 int score_layer_tensor(const mofq_tensor &W, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
-                       mofq_result *res, float *mse_out, void *ws, cudaStream_t st)
+                       const int *fp_formats, mofq_result *res, float *mse_out, void *ws, cudaStream_t st)
 {
     if (int rc = check_tensor(&W)) return rc;
     if (int rc = check_gran(cfg->w_gran, cfg->w_group, W.cols)) return rc;
@@ -130,6 +130,8 @@ int score_layer_tensor(const mofq_tensor &W, const mofq_config *cfg, const CandS
     job.gran = cfg->w_gran;
     job.gran2 = cfg->w_gran2;
     job.group = cfg->w_group;
+    job.fp_formats[0] = fp_formats[0];
+    job.fp_formats[1] = fp_formats[1];
     job.hdr = static_cast<WsHeader *>(ws);
     job.partials = reinterpret_cast<double *>(static_cast<char *>(ws) + sizeof(WsHeader));
     job.fin.mse_out = mse_out;
@@ -231,8 +233,8 @@ int mofq_tensor_error(const mofq_tensor *x, const int32_t *formats, int n, int g
     cfg.w_group = group;
     cfg.metric = MOFQ_TENSOR_MSE;
     CandSet cs;
-    int perm[MOFQ_MAX_CAND], nc;
-    if (int rc = build_candset(formats, n, d0.bits, &cs, perm, &nc)) return rc;
+    int perm[MOFQ_MAX_CAND], nc, fp_formats[2];
+    if (int rc = build_candset(formats, n, d0.bits, &cs, perm, &nc, fp_formats)) return rc;
     if (int rc = check_gran(gran, group, x->cols)) return rc;
     if (gran2 != MOFQ_GRAN_NONE) {
         if (int rc = check_gran(gran2, group, x->cols)) return rc;
@@ -241,7 +243,7 @@ int mofq_tensor_error(const mofq_tensor *x, const int32_t *formats, int n, int g
     if (int rc = check_ws(workspace, workspace_bytes, mofq_tensor_workspace_bytes(x))) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
-    return score_layer_tensor(*x, &cfg, cs, perm, nc, nullptr, mse_out, workspace, st);
+    return score_layer_tensor(*x, &cfg, cs, perm, nc, fp_formats, nullptr, mse_out, workspace, st);
 }
 
 int mofq_layer_output_error(const mofq_layer *L, const mofq_config *cfg, float *mse_out, float *nsr_out,
@@ -291,7 +293,7 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
     for (int i = 0; i < n_layers; ++i) {  // Algorithm 1: for layer in model.layers_to_quant
         int rc;
         if (cfg->metric == MOFQ_TENSOR_MSE)
-            rc = score_layer_tensor(layers[i].W, cfg, cs, perm, nc, results_out + (size_t)i * n_sets, nullptr, workspace, st);
+            rc = score_layer_tensor(layers[i].W, cfg, cs, perm, nc, fp_formats, results_out + (size_t)i * n_sets, nullptr, workspace, st);
         else
             rc = layer_metric_run(layers[i], cfg, results_out + i, nullptr, nullptr, workspace, workspace_bytes, st);
         if (rc) return rc;

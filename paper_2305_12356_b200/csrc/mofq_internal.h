@@ -56,6 +56,7 @@ struct ScoreJob {
     mofq_tensor x;
     CandSet cs;
     int gran, gran2, group;    // gran2 = MOFQ_GRAN_NONE or second granularity
+    int fp_formats[2];         // mofq_format held by each canonical FP slot (-1 if unused)
     Finalize fin;
     WsHeader *hdr;
     double *partials;          // kMaxSlots * kMaxAcc doubles

@@ -13,6 +13,7 @@
 #include <algorithm>
 #include <type_traits>
 
+#include "kq_math.cuh"
 #include "mofq_internal.h"
 
 namespace mofq {
@@ -290,26 +291,37 @@ kq_score_groups(const uint16_t *__restrict__ x, long long n_groups, int group, C
 
 // ---- scoring kernel 2: one row per block; per-channel and/or per-group scales ---------------------------
 // The row is staged in shared memory so that the abs-max pass and the scoring pass cost one HBM read.
-// Accumulator order: [first set][second set]; `grp_first` says whether the group set comes first.
+// Work is chunk-strided (a chunk = 8 elements = 16 bytes), so every thread stays busy whatever the row
+// length: pass 1 leaves one abs-max per chunk; the first `groups per row` threads fold 16-byte chunk maxima
+// into group maxima and derive the group scales; a block reduction gives the row scale; pass 2 scores each
+// chunk against its group's scales and/or the row's scales from the same registers.
+// Arithmetic: packed f32x2 and hardware FP converts (kq_math.cuh).  Accumulator order: [first set][second
+// set]; `grp_first` says whether the group set comes first.
 constexpr int kRowThreads = 256;
 
-template <int DT, int NI, int NFP, bool CH, bool GRP>
+struct RowQ {
+    float q[3];  // abs-max target per canonical slot
+};
+
+template <int DT, int NI, int K0, int K1, bool CH, bool GRP>
 __global__ void __launch_bounds__(kRowThreads)
-kq_score_rows(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, int group, int grp_first,
-              CandSet cs, WsHeader *hdr, double *partials, Finalize fin)
+kq_score_rows(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, int group, int grp_first, RowQ rq,
+              WsHeader *hdr, double *partials, Finalize fin)
 {
-    constexpr int NC = NI + NFP;
+    using S = kqmath::Scorer<DT, NI, K0, K1>;
+    constexpr int NC = S::NC;
     constexpr int NA = NC * ((CH ? 1 : 0) + (GRP ? 1 : 0));
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ double red[33 * NA];
     __shared__ uint32_t mred[34];
-    __shared__ Scales<NC> row_sc;
+    __shared__ kqmath::Sc<NC> row_sc;
     __shared__ int row_status;
     const int chunks = cols >> 3;
-    const int cpg = GRP ? (group >> 3) : 1;
+    const int cpg_shift = GRP ? 31 - __clz(group >> 3) : 0;  // chunks per group is a power of two
     const int gpr = GRP ? cols / group : 0;
-    uint16_t *gmax = reinterpret_cast<uint16_t *>(smem + (size_t)cols * 2);  // per-group abs-max patterns
     const uint4 *row4 = reinterpret_cast<const uint4 *>(smem);
+    uint16_t *cmax = reinterpret_cast<uint16_t *>(smem + (size_t)cols * 2);                               // per-chunk abs-max
+    kqmath::Sc<NC> *gsc = reinterpret_cast<kqmath::Sc<NC> *>(smem + (size_t)cols * 2 + (((size_t)chunks * 2 + 15) & ~(size_t)15));
     double dacc[NA];
 #pragma unroll
     for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
@@ -320,63 +332,68 @@ kq_score_rows(const uint16_t *__restrict__ x, long long rows, int cols, long lon
         for (int q = threadIdx.x; q < chunks; q += kRowThreads) cp_async16(smem + q * 16, src + (size_t)q * 16);
         cp_async_wait_all();
         __syncthreads();
-        // pass 1: abs-max
+        // pass 1: abs-max per chunk
         uint32_t m16 = 0;
-        if (GRP) {
-            for (int g = threadIdx.x; g < gpr; g += kRowThreads) {
-                const uint4 *base = row4 + g * cpg;
-                uint32_t m = 0;
-                for (int j = 0; j < cpg; ++j) m = absmax_chunk(base[(j + g) & (cpg - 1)], m);
-                const uint32_t gm = fold16(m);
-                gmax[g] = (uint16_t)gm;
-                m16 = max(m16, gm);
-            }
-        } else {
-            uint32_t m = 0;
-            for (int q = threadIdx.x; q < chunks; q += kRowThreads) m = absmax_chunk(row4[q], m);
-            m16 = fold16(m);
+        for (int q = threadIdx.x; q < chunks; q += kRowThreads) {
+            const uint32_t c16 = kqmath::fold16(kqmath::absmax_chunk<DT>(row4[q], 0u));
+            if (GRP) cmax[q] = (uint16_t)c16;
+            m16 = max(m16, c16);
         }
-        if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+        if (kqmath::mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+        if (GRP) {
+            __syncthreads();
+            for (int g = threadIdx.x; g < gpr; g += kRowThreads) {
+                uint32_t gm = 0;
+                for (int j = 0; j < (1 << cpg_shift); ++j) gm = max(gm, (uint32_t)cmax[(g << cpg_shift) + j]);
+                const float a = kqmath::mag16_to_float<DT>(gm);
+                kqmath::Sc<NC> sc;
+#pragma unroll
+                for (int j = 0; j < NC; ++j) kqmath::scale_pair(a, rq.q[j], sc.s[j], sc.inv[j], status);
+                gsc[g] = sc;
+            }
+        }
         if (CH) {
             const uint32_t rm = block_max_u32(m16, mred);
             if (threadIdx.x == 0) {
                 int st = 0;
-                make_scales<NI, NFP>(mag16_to_float<DT>(rm), cs, row_sc, st);
+                kqmath::Sc<NC> sc;
+#pragma unroll
+                for (int j = 0; j < NC; ++j) kqmath::scale_pair(kqmath::mag16_to_float<DT>(rm), rq.q[j], sc.s[j], sc.inv[j], st);
+                row_sc = sc;
                 row_status = st;
             }
             __syncthreads();
             status |= row_status;
+        } else {
+            __syncthreads();
         }
         // pass 2: score
-        float acc_g[NC], acc_c[NC];  // group-scale and channel-scale candidates
-#pragma unroll
-        for (int j = 0; j < NC; ++j) acc_g[j] = acc_c[j] = 0.0f;
-        if (GRP) {
-            Scales<NC> rsc;
-            if (CH) rsc = row_sc;
-            for (int g = threadIdx.x; g < gpr; g += kRowThreads) {
-                const uint4 *base = row4 + g * cpg;
-                Scales<NC> gsc;
-                make_scales<NI, NFP>(mag16_to_float<DT>(gmax[g]), cs, gsc, status);
-                for (int j = 0; j < cpg; ++j) {
-                    const uint4 v = base[(j + g) & (cpg - 1)];
-                    score_chunk<DT, NI, NFP>(v, gsc, cs, acc_g);
-                    if (CH) score_chunk<DT, NI, NFP>(v, rsc, cs, acc_c);
-                }
+        S sg, sc;
+        sg.clear();
+        sc.clear();
+        if (CH) sc.set_scales(row_sc);
+        for (int q = threadIdx.x; q < chunks; q += kRowThreads) {
+            const uint4 v = row4[q];
+            if (GRP) {
+                sg.set_scales(gsc[q >> cpg_shift]);
+                sg.chunk(v);
             }
-        } else {
-            const Scales<NC> rsc = row_sc;
-            for (int q = threadIdx.x; q < chunks; q += kRowThreads) score_chunk<DT, NI, NFP>(row4[q], rsc, cs, acc_c);
+            if (CH) sc.chunk(v);
         }
+        double a_g[NC], a_c[NC];
+#pragma unroll
+        for (int j = 0; j < NC; ++j) a_g[j] = a_c[j] = 0.0;
+        if (GRP) sg.end(a_g);
+        if (CH) sc.end(a_c);
         if (CH && GRP) {
 #pragma unroll
             for (int j = 0; j < NC; ++j) {
-                dacc[j] += (double)(grp_first ? acc_g[j] : acc_c[j]);
-                dacc[NC + j] += (double)(grp_first ? acc_c[j] : acc_g[j]);
+                dacc[j] += grp_first ? a_g[j] : a_c[j];
+                dacc[NC + j] += grp_first ? a_c[j] : a_g[j];
             }
         } else {
 #pragma unroll
-            for (int j = 0; j < NC; ++j) dacc[j] += (double)(GRP ? acc_g[j] : acc_c[j]);
+            for (int j = 0; j < NC; ++j) dacc[j] += GRP ? a_g[j] : a_c[j];
         }
         __syncthreads();
     }
@@ -797,24 +814,42 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
 
     // row kernel: per-channel, per-group on a strided tensor, or both from one read
     if (x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
+    const int chunks = (int)(x.cols / 8);
     const int gpr = has_grp ? (int)(x.cols / job.group) : 0;
-    const size_t smem = (size_t)x.cols * 2 + (size_t)((gpr * 2 + 15) & ~15);
+    const size_t smem = (size_t)x.cols * 2 + (((size_t)chunks * 2 + 15) & ~(size_t)15) + (size_t)gpr * 8 * 3 + 16;
     if (smem > 200 * 1024) return MOFQ_ERR_UNSUPPORTED;
     const int grp_first = (job.gran == MOFQ_PER_GROUP) ? 1 : 0;
-    return dispatch_cands(x.dtype, job.cs.n_int, job.cs.n_fp, [&](auto DT, auto NI, auto NFP) {
-        auto launch = [&](auto kernel) {
-            if (int rc = set_smem(kernel, smem)) return rc;
-            const int occ = std::max(1, blocks_per_sm((const void *)kernel, kRowThreads, smem));
-            const int grid = (int)std::min<long long>(x.rows, std::min<long long>((long long)nsm * occ, kMaxSlots));
-            kernel<<<grid, kRowThreads, smem, st>>>(xp, x.rows, (int)x.cols, x.ld, has_grp ? job.group : 8, grp_first, job.cs,
-                                                    job.hdr, job.partials, job.fin);
-            MOFQ_CUDA_OK(cudaGetLastError());
-            return MOFQ_OK;
-        };
-        if (has_ch && has_grp) return launch(kq_score_rows<DT(), NI(), NFP(), true, true>);
-        if (has_ch) return launch(kq_score_rows<DT(), NI(), NFP(), true, false>);
-        return launch(kq_score_rows<DT(), NI(), NFP(), false, true>);
-    });
+    RowQ rq{};
+    if (job.cs.n_int) rq.q[0] = job.cs.int_q;
+    for (int f = 0; f < job.cs.n_fp; ++f) rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
+    auto kind = [](int format) {
+        return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
+    };
+    const int k0 = job.cs.n_fp > 0 ? kind(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? kind(job.fp_formats[1]) : -1;
+    auto launch = [&](auto kernel) {
+        if (int rc = set_smem(kernel, smem)) return rc;
+        const int occ = std::max(1, blocks_per_sm((const void *)kernel, kRowThreads, smem));
+        const int grid = (int)std::min<long long>(x.rows, std::min<long long>((long long)nsm * occ, kMaxSlots));
+        kernel<<<grid, kRowThreads, smem, st>>>(xp, x.rows, (int)x.cols, x.ld, has_grp ? job.group : 8, grp_first, rq, job.hdr,
+                                                job.partials, job.fin);
+        MOFQ_CUDA_OK(cudaGetLastError());
+        return MOFQ_OK;
+    };
+#define MOFQ_ROWS(DT_, NI_, K0_, K1_)                                                                   \
+    if (x.dtype == DT_ && job.cs.n_int == NI_ && k0 == K0_ && k1 == K1_) {                              \
+        if (has_ch && has_grp) return launch(kq_score_rows<DT_, NI_, K0_, K1_, true, true>);            \
+        if (has_ch) return launch(kq_score_rows<DT_, NI_, K0_, K1_, true, false>);                      \
+        return launch(kq_score_rows<DT_, NI_, K0_, K1_, false, true>);                                  \
+    }
+#define MOFQ_ROWS_DT(DT_)                                                                                        \
+    MOFQ_ROWS(DT_, 1, -1, -1) MOFQ_ROWS(DT_, 0, 0, -1) MOFQ_ROWS(DT_, 1, 0, -1) MOFQ_ROWS(DT_, 0, 0, 0) MOFQ_ROWS(DT_, 1, 0, 0) \
+    MOFQ_ROWS(DT_, 0, 1, -1) MOFQ_ROWS(DT_, 1, 1, -1) MOFQ_ROWS(DT_, 0, 2, -1) MOFQ_ROWS(DT_, 1, 2, -1)                         \
+    MOFQ_ROWS(DT_, 0, 1, 2) MOFQ_ROWS(DT_, 1, 1, 2) MOFQ_ROWS(DT_, 0, 2, 1) MOFQ_ROWS(DT_, 1, 2, 1)
+    MOFQ_ROWS_DT(0)
+    MOFQ_ROWS_DT(1)
+#undef MOFQ_ROWS_DT
+#undef MOFQ_ROWS
+    return MOFQ_ERR_UNSUPPORTED;
 }
 
 // Per-channel abs-max scales; codes (and scales) of n formats from one read.  formats[i] is a mofq_format.

@@ -23,6 +23,7 @@
 #include <type_traits>
 #include <vector>
 
+#include "kq_math.cuh"
 #include "mofq_internal.h"
 
 namespace mofq {
@@ -34,30 +35,8 @@ constexpr int kConsumerWarps = 4;
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kThreads = kConsumers + 32;  // + one producer warp
 constexpr long long kWaitCycles = 4000000000LL;  // ~2 s: a wait that long means the pipeline is broken
-constexpr float kMagic = 12582912.0f;
+using namespace kqmath;
 
-enum { FPK_E2M1 = 0, FPK_E4M3 = 1, FPK_E5M2 = 2 };
-
-// ---- PTX wrappers -------------------------------------------------------------------------------------
-__device__ __forceinline__ uint64_t pk(float lo, float hi) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
-__device__ __forceinline__ void upk(uint64_t v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { uint64_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) { uint64_t d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
-
-// two non-negative floats -> FP4/FP8 pair (RNE, saturating) -> the same two values as f16x2
-template <int KIND>
-__device__ __forceinline__ uint32_t fp_round_trip(float lo, float hi)
-{
-    uint32_t h2;
-    if (KIND == FPK_E2M1)
-        asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %2, %1; cvt.rn.f16x2.e2m1x2 %0, t; }" : "=r"(h2) : "f"(lo), "f"(hi));
-    else if (KIND == FPK_E4M3)
-        asm("{ .reg .b16 t; cvt.rn.satfinite.e4m3x2.f32 t, %2, %1; cvt.rn.f16x2.e4m3x2 %0, t; }" : "=r"(h2) : "f"(lo), "f"(hi));
-    else
-        asm("{ .reg .b16 t; cvt.rn.satfinite.e5m2x2.f32 t, %2, %1; cvt.rn.f16x2.e5m2x2 %0, t; }" : "=r"(h2) : "f"(lo), "f"(hi));
-    return h2;
-}
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t *bar, int count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count)); }
@@ -92,124 +71,6 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t b
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-// ---- per-format scoring --------------------------------------------------------------------------------
-template <int NC>
-struct Sc {
-    float s[NC], inv[NC];
-};
-
-__device__ __forceinline__ void scale_pair(float a, float Q, float &s, float &inv, int &status)
-{
-    if (a == 0.0f) {
-        s = 1.0f;
-        inv = 1.0f;
-    } else {
-        s = __fdiv_rn(a, Q);
-        inv = __fdiv_rn(Q, a);
-        if (isinf(inv)) status |= MOFQ_STATUS_SCALE_OVERFLOW;
-    }
-}
-
-// magnitudes of the two 16-bit values in w, as packed binary32
-template <int DT>
-__device__ __forceinline__ uint64_t abs_unpack(uint32_t w)
-{
-    const uint32_t wa = w & 0x7FFF7FFFu;
-    if (DT == MOFQ_F16) {
-        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&wa));
-        return pk(f.x, f.y);
-    }
-    return pk(__uint_as_float(wa << 16), __uint_as_float(wa & 0xFFFF0000u));
-}
-
-template <int DT>
-__device__ __forceinline__ uint32_t absmax_chunk(const uint4 v, uint32_t m)
-{
-    if (DT == MOFQ_F16) {
-        __half2 mm = *reinterpret_cast<__half2 *>(&m);
-        mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __half2 *>(&v.x)));
-        mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __half2 *>(&v.y)));
-        mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __half2 *>(&v.z)));
-        mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __half2 *>(&v.w)));
-        return *reinterpret_cast<uint32_t *>(&mm);
-    }
-    __nv_bfloat162 mm = *reinterpret_cast<__nv_bfloat162 *>(&m);
-    mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&v.x)));
-    mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&v.y)));
-    mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&v.z)));
-    mm = __hmax2_nan(mm, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&v.w)));
-    return *reinterpret_cast<uint32_t *>(&mm);
-}
-
-// fold the two 16-bit lanes of a packed abs-max; NaN patterns (> Inf) stay on top as integers
-__device__ __forceinline__ uint32_t fold16(uint32_t m) { return max(m & 0x7FFFu, (m >> 16) & 0x7FFFu); }
-
-template <int DT>
-__device__ __forceinline__ float mag16_to_float(uint32_t m16)
-{
-    if (DT == MOFQ_F16) return __half2float(__ushort_as_half((unsigned short)m16));
-    return __uint_as_float(m16 << 16);
-}
-template <int DT>
-__device__ __forceinline__ bool mag16_nonfinite(uint32_t m16)
-{
-    return m16 >= (DT == MOFQ_F16 ? 0x7C00u : 0x7F80u);
-}
-
-template <int DT, int NI, int K0, int K1>  // K0/K1: FP kind of slot 0/1, or -1
-struct Scorer {
-    static constexpr int NFP = (K0 >= 0) + (K1 >= 0);
-    static constexpr int NC = NI + NFP;
-    uint64_t inv2[NC], ns2[NC], acc2[NC];
-
-    __device__ __forceinline__ void begin(const Sc<NC> &sc)
-    {
-#pragma unroll
-        for (int j = 0; j < NC; ++j) {
-            inv2[j] = pk(sc.inv[j], sc.inv[j]);
-            ns2[j] = pk(-sc.s[j], -sc.s[j]);
-            acc2[j] = 0;
-        }
-    }
-    template <int KIND>
-    __device__ __forceinline__ void fp_slot(int j, uint64_t a2)
-    {
-        float tl, th;
-        upk(mul2(a2, inv2[j]), tl, th);
-        const uint32_t h2 = fp_round_trip<KIND>(tl, th);
-        const float2 rf = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
-        const uint64_t e2 = fma2(pk(rf.x, rf.y), ns2[j], a2);
-        acc2[j] = fma2(e2, e2, acc2[j]);
-    }
-    __device__ __forceinline__ void word(uint32_t w)
-    {
-        const uint64_t a2 = abs_unpack<DT>(w);
-        if (NI) {
-            const uint64_t mg = pk(kMagic, kMagic), nmg = pk(-kMagic, -kMagic);
-            const uint64_t r2 = add2(fma2(a2, inv2[0], mg), nmg);
-            const uint64_t e2 = fma2(r2, ns2[0], a2);
-            acc2[0] = fma2(e2, e2, acc2[0]);
-        }
-        if (K0 >= 0) fp_slot<K0 >= 0 ? K0 : 0>(NI, a2);
-        if (K1 >= 0) fp_slot<K1 >= 0 ? K1 : 0>(NI + 1, a2);
-    }
-    __device__ __forceinline__ void chunk(const uint4 v)
-    {
-        word(v.x);
-        word(v.y);
-        word(v.z);
-        word(v.w);
-    }
-    __device__ __forceinline__ void end(double *dacc)
-    {
-#pragma unroll
-        for (int j = 0; j < NC; ++j) {
-            float lo, hi;
-            upk(acc2[j], lo, hi);
-            dacc[j] += (double)(lo + hi);
-        }
-    }
-};
 
 // ---- the kernel ---------------------------------------------------------------------------------------
 struct MtParams {
