@@ -212,6 +212,13 @@ int mofq_tensor_error_noalloc(const mofq_tensor *x, const int32_t *formats, int 
                               float *mse_out, int32_t *status_out, void *stream);
 size_t mofq_noalloc_scratch_bytes(void);
 
+/*
+ * mofq_diag_fp_round - diagnostic: rounds n binary32 values onto the unscaled FP grid (Section 2, Table 3) exactly as
+ * the scoring kernels do (hardware convert, round-to-nearest-even, saturating at the grid maximum) and writes the
+ * grid values.  format: MOFQ_FP4_E2M1, MOFQ_FP8_E4M3 or MOFQ_FP8_E5M2.  t, out: device, n floats.
+ */
+int mofq_diag_fp_round(int format, const float *t, float *out, int64_t n, void *stream);
+
 /* Workspace sizes in bytes (host-side arithmetic only). */
 size_t mofq_tensor_workspace_bytes(const mofq_tensor *x);
 size_t mofq_workspace_bytes(const mofq_layer *layers, int n_layers, const mofq_config *cfg);

@@ -73,6 +73,8 @@ def lib():
                                                 vp, vp, vp]
         L.mofq_noalloc_scratch_bytes.restype = sz
         L.mofq_noalloc_scratch_bytes.argtypes = []
+        L.mofq_diag_fp_round.restype = C.c_int
+        L.mofq_diag_fp_round.argtypes = [C.c_int, vp, vp, C.c_int64, vp]
         L.mofq_layer_output_error.restype = C.c_int
         L.mofq_layer_output_error.argtypes = [C.POINTER(MofqLayer), C.POINTER(MofqConfig), vp, vp, vp, sz, vp]
         for name in ("mofq_select_formats", "mofq_select_formats_host"):
@@ -237,6 +239,14 @@ def tensor_error_noalloc(x, formats, gran, gran2=None, group=0, mse_out=None, st
     _check(L.mofq_tensor_error_noalloc(C.byref(d), fm, n, _gran(gran), g2, group, mse_out.data_ptr(),
                                        status_out.data_ptr(), _stream(x.device)))
     return mse_out, status_out
+
+
+def diag_fp_round(fmt, t):
+    """mofq_diag_fp_round: the scoring kernels' FP grid rounding applied to a float32 CUDA tensor."""
+    t = t.contiguous().float()
+    out = torch.empty_like(t)
+    _check(lib().mofq_diag_fp_round(_fmt(fmt), t.data_ptr(), out.data_ptr(), t.numel(), _stream(t.device)))
+    return out
 
 
 def layer_output_error(X, W, cfg, workspace=None):

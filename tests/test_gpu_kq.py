@@ -286,3 +286,27 @@ def test_multi_tensor_path_status_per_layer(dev):
     cfg = mofq.make_config(4, ["INT4", "FP4_E2M1"], w_gran="group", w_group=128)
     recs = mofq.select_formats(layers, cfg)
     assert [bool(r["status"] & B.STATUS_NONFINITE_INPUT) for r in recs] == [False, False, True, False]
+
+
+# ---- the hardware converts used by the scoring kernels round like the definition ------------------------------------------
+@pytest.mark.parametrize("name", ["FP4_E2M1", "FP8_E4M3", "FP8_E5M2"])
+def test_hardware_fp_rounding_matches_oracle(orc, dev, name):
+    fmt = getattr(orc, name)
+    half = 2 ** (orc.format_bits(fmt) - 1)
+    pos = orc.decode_table(fmt)[:half]
+    pos = pos[~np.isnan(pos)]
+    mids = (pos[:-1] + pos[1:]) / 2
+    pts = [pos, mids]
+    for d in (-2, -1, 1, 2):                                                   # neighbours of every tie in binary32
+        pts.append((mids.astype(np.float32).view(np.uint32).astype(np.int64) + d).astype(np.uint32).view(np.float32).astype(np.float64))
+    g = np.random.default_rng(9)
+    pts.append(g.uniform(0, pos[-1] * 1.5, 20000))
+    pts.append(np.exp(g.uniform(np.log(pos[1] / 64), np.log(pos[-1] * 2), 20000)))
+    t = np.concatenate(pts).astype(np.float32)
+    t = np.concatenate([t, -t, np.array([0.0, -0.0, 1e30, -1e30], np.float32)])
+    from paper_2305_12356_b200.binding import diag_fp_round
+    got = diag_fp_round(name, torch.from_numpy(t).to(dev)).cpu().numpy()
+    tab = orc.decode_table(fmt)
+    want = np.array([tab[orc.encode_fp_arith(fmt, v)] for v in t])
+    np.testing.assert_array_equal(got.astype(np.float64), want)
+    np.testing.assert_array_equal(np.signbit(got), np.signbit(t))               # the sign survives rounding to zero
