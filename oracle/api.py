@@ -23,7 +23,8 @@ _lib = None
 def lib():
     global _lib
     if _lib is None:
-        L = C.CDLL(build())
+        import os
+        L = C.CDLL(os.environ.get("MOFQ_ORACLE_LIB") or build())   # the override serves the mutation test only
         u16p, u8p, f32p, f64p = (C.POINTER(t) for t in (C.c_uint16, C.c_uint8, C.c_float, C.c_double))
         i64 = C.c_int64
         L.orc_format_bits.restype = C.c_int
