@@ -241,8 +241,8 @@ def main():
         wbuf = torch.empty(max_w, dtype=torch.float16, device=dev)
         xbuf = torch.empty(max_x, dtype=torch.bfloat16, device=dev)
         views = [(wbuf[:o * i].view(o, i), xbuf[:T * i].view(T, i)) for _, o, i in shapes]
-        big = max(views, key=lambda v: v[0].numel())
-        ws = torch.empty(mofq.workspace_bytes([big], cfg), dtype=torch.uint8, device=dev)
+        distinct = {tuple(v[0].shape): v for v in views}
+        ws = torch.empty(max(mofq.workspace_bytes([v], cfg) for v in distinct.values()), dtype=torch.uint8, device=dev)
         preps = [mofq.prepare_layers([v]) for v in views]
         res_views = [results[li * B.RESULT_BYTES:(li + 1) * B.RESULT_BYTES] for li in range(len(shapes))]
 

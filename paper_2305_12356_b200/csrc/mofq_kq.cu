@@ -699,6 +699,36 @@ kq_emit_codes_rows(const uint16_t *__restrict__ x, long long rows, int cols, lon
     if (status) atomicOr(&hdr->status, status);
 }
 
+// per-tensor variant: the abs-max is already in the workspace header; codes of every requested format from one read
+template <int DT>
+__global__ void __launch_bounds__(256)
+kq_emit_codes_uniform(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, EmitSet es, WsHeader *hdr)
+{
+    int status = 0;
+    const uint32_t m16 = *reinterpret_cast<volatile uint32_t *>(&hdr->absmax_bits);
+    if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+    float inv[3];
+    for (int f = 0; f < es.n; ++f) {
+        float s;
+        scale_pair(mag16_to_float<DT>(m16), es.Q[f], s, inv[f], status);
+        if (blockIdx.x == 0 && threadIdx.x == 0 && es.scales[f]) es.scales[f][0] = s;
+    }
+    const long long total = rows * chunks_per_row;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / chunks_per_row;
+        const int c = (int)(i - r * chunks_per_row);
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c);
+        for (int f = 0; f < es.n; ++f) {
+            const int fmt = es.format[f];
+            const bool four = fmt == MOFQ_INT4 || fmt == MOFQ_FP4_E2M1 || fmt == MOFQ_FP4_E2M1_IEEE;
+            const uint64_t cd = codes8<DT>(v, fmt, inv[f]);
+            if (four) reinterpret_cast<uint32_t *>(es.codes[f])[i] = (uint32_t)cd;
+            else reinterpret_cast<uint2 *>(es.codes[f])[i] = make_uint2((uint32_t)cd, (uint32_t)(cd >> 32));
+        }
+    }
+    if (status) atomicOr(&hdr->status, status);
+}
+
 // ---- host-side dispatch ----------------------------------------------------------------------------------
 #define MOFQ_CUDA_OK(expr)                      \
     do {                                        \
@@ -850,6 +880,32 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
 #undef MOFQ_ROWS_DT
 #undef MOFQ_ROWS
     return MOFQ_ERR_UNSUPPORTED;
+}
+
+// Per-tensor scale from the abs-max already stored in hdr->absmax_bits (launch_absmax); codes of n formats from one read.
+int launch_emit_codes_uniform(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
+                              WsHeader *hdr, cudaStream_t st)
+{
+    if (n < 1 || n > 3 || x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+    EmitSet es{};
+    es.n = n;
+    for (int i = 0; i < n; ++i) {
+        FmtDesc d;
+        if (!describe_format(formats[i], &d)) return MOFQ_ERR_INVALID_ARG;
+        es.format[i] = formats[i];
+        es.Q[i] = d.Q;
+        es.codes[i] = static_cast<unsigned char *>(codes[i]);
+        es.scales[i] = scales ? scales[i] : nullptr;
+    }
+    const uint16_t *xp = static_cast<const uint16_t *>(x.data);
+    const long long total = x.rows * (x.cols / 8);
+    const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
+    if (x.dtype == MOFQ_F16)
+        kq_emit_codes_uniform<0><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, es, hdr);
+    else
+        kq_emit_codes_uniform<1><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, es, hdr);
+    MOFQ_CUDA_OK(cudaGetLastError());
+    return MOFQ_OK;
 }
 
 // Per-channel abs-max scales; codes (and scales) of n formats from one read.  formats[i] is a mofq_format.

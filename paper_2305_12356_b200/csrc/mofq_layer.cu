@@ -444,7 +444,7 @@ LayerWs layer_ws_layout(long long T, long long n_in, long long n_out)
     LayerWs w{};
     size_t off = 0;
     w.x16 = off; off += align256((size_t)T * n_in * 2);
-    w.cx = off;  off += align256((size_t)T * n_in * 2);
+    w.cx = off;  off += 3 * align256((size_t)T * n_in);        // 8-bit codes of up to 3 formats, or 16-bit values of one
     w.cw = off;  off += 3 * align256((size_t)n_out * n_in);   // 8-bit codes of up to 3 formats, or 16-bit values of one
     w.y = off;   off += align256((size_t)T * n_out * 4);
     w.sw = off;  off += 3 * align256((size_t)n_out * 4);
@@ -547,9 +547,13 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
     // reference operand for X (and its abs-max, which also serves the per-tensor activation scale)
     const void *xa = X.data;
     long long xa_ld = X.ld;
-    if (X.dtype != op_dtype) {  // bf16 activations with fp16 weights
+    const bool native8 = !cfg->is_w_only && cfg->bit_width == 8 && (n_in % 16) == 0;
+    const bool fused = native8 && cfg->n_candidates <= 3;
+    if (X.dtype != op_dtype || fused) {  // one abs-max of X serves the exact fp16 copy and the per-tensor activation scales
         if (cudaMemsetAsync(&hdr->absmax_bits, 0, sizeof(uint32_t), st) != cudaSuccess) return MOFQ_ERR_CUDA;
         if (int rc = launch_absmax(X, hdr, st)) return rc;
+    }
+    if (X.dtype != op_dtype) {  // bf16 activations with fp16 weights
         const long long total = T * (n_in / 8);
         const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
         x_bf16_to_f16<<<grid, 256, 0, st>>>(static_cast<const uint16_t *>(X.data), T, (int)n_in, X.ld, hdr, x16, scal);
@@ -561,9 +565,9 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
         if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
     }
     // WA with 8-bit candidates: the codes themselves are the tensor-core operands (int8 / e4m3 / e5m2 kinds)
-    const bool native8 = !cfg->is_w_only && cfg->bit_width == 8 && (n_in % 16) == 0;
     // native path: the codes of every candidate from one read of W (one byte per element and format)
-    const bool fused_w = native8 && cfg->n_candidates <= 3;
+    const bool fused_w = fused;
+    const size_t cx_stride = align256((size_t)T * n_in);
     const size_t cw_stride = align256((size_t)n_out * n_in), sw_stride = align256((size_t)n_out * 4) / 4;
     if (fused_w) {
         void *cptr[3];
@@ -575,6 +579,11 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
             fmts[i] = cfg->candidates[i];
         }
         if (int rc = launch_emit_codes_rows(W, cfg->n_candidates, fmts, cptr, sptr, hdr, st)) return rc;
+        for (int i = 0; i < cfg->n_candidates; ++i) {  // activations: codes of every candidate, scales in scal[1 + i]
+            cptr[i] = reinterpret_cast<unsigned char *>(cx) + (size_t)i * cx_stride;
+            sptr[i] = scal + 1 + i;
+        }
+        if (int rc = launch_emit_codes_uniform(X, cfg->n_candidates, fmts, cptr, sptr, hdr, st)) return rc;
     }
     int grid_used = 0, max_grid = 0;
     if (int rc = run_gemm(xa, T, xa_ld, W.data, n_out, W.ld, n_in, op_dtype, 0, Y, scal, nullptr, partials, &hdr->status, &grid_used, st))
@@ -592,7 +601,11 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
         const void *a = xa;
         long long a_ld = xa_ld;
         const float *alpha = scal;
-        if (!cfg->is_w_only) {
+        if (fused) {
+            a = reinterpret_cast<unsigned char *>(cx) + (size_t)i * cx_stride;
+            a_ld = n_in;
+            alpha = scal + 1 + i;
+        } else if (!cfg->is_w_only) {
             if (int rc = launch_emit(X, fd[i], MOFQ_PER_TENSOR, 0, nullptr, native8 ? cx : nullptr, scal + 1, nullptr,
                                      native8 ? nullptr : cx, op_dtype, hdr, st))
                 return rc;
