@@ -237,8 +237,21 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             tc_fence_after();
             const int row = m0 + q * 32 + lane;
             float fsum = 0.0f;
+            // the stored Y of the next 32-column chunk is fetched while the current chunk is processed
+            const bool vec = (p.N & 3) == 0;
+            float4 ycur[8], ynext[8];
+            auto prefetch_y = [&](int c, float4 (&y)[8]) {
+                const int pc0 = n0 + c * 32;
+                if (p.mode == 1 && row < p.M && vec && pc0 + 32 <= p.N) {
+                    const float4 *src = reinterpret_cast<const float4 *>(p.Y + (size_t)row * p.N + pc0);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) y[j] = __ldg(src + j);
+                }
+            };
+            prefetch_y(0, ycur);
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
+                if (c + 1 < BN / 32) prefetch_y(c + 1, ynext);
                 uint32_t r[32];
                 tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), r);
                 const int col0 = n0 + c * 32;
@@ -248,7 +261,7 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 }
                 if (row < p.M) {
                     float *yrow = p.Y + (size_t)row * p.N + col0;
-                    if (col0 + 32 <= p.N && (p.N & 3) == 0) {
+                    if (col0 + 32 <= p.N && vec) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             float4 v;
@@ -263,7 +276,7 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                                 fsum = fmaf(v.z, v.z, fsum);
                                 fsum = fmaf(v.w, v.w, fsum);
                             } else {
-                                const float4 y = *reinterpret_cast<const float4 *>(yrow + j);
+                                const float4 y = ycur[j >> 2];
                                 float4 cs = make_float4(1.f, 1.f, 1.f, 1.f);
                                 if (p.col_scale) cs = __ldg(reinterpret_cast<const float4 *>(p.col_scale + col0 + j));
                                 const float d0 = y.x - __uint_as_float(r[j]) * (alpha * cs.x);
@@ -291,6 +304,8 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         }
                     }
                 }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) ycur[j] = ynext[j];
             }
             dsum += (double)fsum;
             tc_fence_before();
