@@ -368,7 +368,8 @@ kq_score_rows(const uint16_t *__restrict__ x, long long rows, int cols, long lon
             __syncthreads();
         }
         // pass 2: score
-        S sg, sc;
+        S sg;                                            // group scales change from chunk to chunk: unscaled accumulation
+        kqmath::Scorer<DT, NI, K0, K1, true> sc;         // the row's scales are fixed: scaled accumulation
         sg.clear();
         sc.clear();
         if (CH) sc.set_scales(row_sc);

@@ -14,7 +14,8 @@
 //         one binary32 ulp of a tie, and at a tie both neighbours have the same error, so the
 //         squared-error sum agrees with the two-rounding definition far inside the 1e-5 tolerance.
 //   FP  : t = RN32(a*inv); r = hardware convert of t to the 4/8-bit float (round-to-nearest-even,
-//         saturating) and back; e = fma(-r, s, a); sum += e*e.
+//         saturating) and back to f16; d = r - t with a mixed-precision subtract; the group's sum of d*d is
+//         multiplied by scale^2 once per group (the scale is fixed over a lane's group).
 // Packed two-lane binary32 instructions (f32x2) halve the issue slots of the multiply/add work.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -99,7 +100,7 @@ template <int DT, int NI, int K0, int K1>
 __global__ void __launch_bounds__(kThreads)
 kq_score_mt(const MtParams p)
 {
-    using S = Scorer<DT, NI, K0, K1>;
+    using S = Scorer<DT, NI, K0, K1, true>;
     constexpr int NC = S::NC;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages];
