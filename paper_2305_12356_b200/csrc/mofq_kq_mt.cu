@@ -199,8 +199,13 @@ kq_score_mt(const MtParams p)
         for (int g = threadIdx.x; g < ng; g += kConsumers) {
             const uint4 *base = tile + g * cpg;
             uint32_t m = 0;
+            if (cpg == 16) {  // group of 128: fully unrolled
+#pragma unroll
+                for (int j = 0; j < 16; ++j) m = absmax_chunk<DT>(base[(j + g) & 15], m);
+            } else {
 #pragma unroll 4
-            for (int j = 0; j < cpg; ++j) m = absmax_chunk<DT>(base[(j + g) & (cpg - 1)], m);
+                for (int j = 0; j < cpg; ++j) m = absmax_chunk<DT>(base[(j + g) & (cpg - 1)], m);
+            }
             const uint32_t m16 = fold16(m);
             if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
             const float a = mag16_to_float<DT>(m16);
@@ -209,8 +214,13 @@ kq_score_mt(const MtParams p)
             for (int j = 0; j < NC; ++j) scale_pair(a, p.q[j], sc.s[j], sc.inv[j], status);
             S scorer;
             scorer.begin(sc);
+            if (cpg == 16) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) scorer.chunk(base[(j + g) & 15]);
+            } else {
 #pragma unroll 4
-            for (int j = 0; j < cpg; ++j) scorer.chunk(base[(j + g) & (cpg - 1)]);
+                for (int j = 0; j < cpg; ++j) scorer.chunk(base[(j + g) & (cpg - 1)]);
+            }
             scorer.end(dacc);
         }
         __syncwarp();
