@@ -28,9 +28,9 @@ if ROOT not in sys.path:
 
 METRIC = "GB/s of fp16 tensor quantized+scored (both formats)"
 UNIT = "GB/s"
-# DRAM bytes per element of kq_score_mt from the ncu capture summarised in profiles/ (read 809.54 MB + write 3.93 MB
+# DRAM bytes per element of kq_score_mt from the ncu capture summarised in profiles/ (read 809.55 MB + write 4.51 MB
 # for 404,750,336 elements on a 14-layer case; traffic is proportional to the elements processed)
-KQ_MT_DRAM_BYTES_PER_ELEMENT = (809.54e6 + 3.93e6) / 404750336
+KQ_MT_DRAM_BYTES_PER_ELEMENT = (809.55e6 + 4.51e6) / 404750336
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
