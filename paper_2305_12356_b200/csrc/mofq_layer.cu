@@ -20,6 +20,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "mofq_internal.h"
 
@@ -33,10 +34,18 @@ constexpr int kRingBytes = 192 * 1024;
 constexpr int kGemmThreads = 192;  // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-5: epilogue
 // Tile width BN is 128 or 256: the wider tile moves 25% fewer operand bytes per flop (the main loop is bound by
 // L2 -> shared-memory traffic), the narrower one quantises better onto 148 SMs.  Two accumulators of BN columns.
-template <int BN> struct TileCfg {
-    static constexpr int kBBytes = BN * kRowBytes;
-    static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kStages = kRingBytes / kStageBytes;  // 6 (BN=128) or 4 (BN=256)
+// CG = 2: a cluster of two CTAs computes a 256 x BN tile; each CTA stages its own 128 rows of A and BN/2 rows of B
+// (32 KB per k-block for BN = 256 instead of 48 KB), the leader CTA issues M = 256 MMAs that read both CTAs' shared
+// memory and write both CTAs' tensor memory.
+// KA = K atoms (128-byte swizzle rows) per stage: with KA = 2 one barrier wait and one commit serve 8 MMAs instead of
+// 4, which halves the per-stage overhead of the issuing thread (measured: ~400 cycles per stage that tensor execution
+// does not hide).
+template <int BN, int CG = 1> struct TileCfg {
+    static constexpr int kBRows = BN / CG;                    // rows of B staged by one CTA
+    static constexpr int kBBytes = kBRows * kRowBytes;        // one K atom of B
+    static constexpr int KA = (kABytes + kBBytes) <= 32 * 1024 ? 2 : 1;
+    static constexpr int kStageBytes = KA * (kABytes + kBBytes);
+    static constexpr int kStages = kRingBytes / kStageBytes;  // 3 (64 KB stages) or 4 (48 KB stages)
     static constexpr int kTmemCols = 2 * BN;
 };
 constexpr long long kWaitCycles = 4000000000LL;
@@ -95,6 +104,48 @@ __device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t a_desc, uint
     asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p; }"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// ---- two-CTA (cta_group::2) forms: a pair of CTAs in a cluster shares one 256-row MMA ----------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load whose completion bytes are counted on the LEADER CTA's barrier (cluster address); no multicast
+__device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, int c0, int c1, uint32_t leader_bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(leader_bar) : "memory");
+}
+// arrive on the barrier at this offset in both CTAs of the pair once the MMAs issued so far have completed
+__device__ __forceinline__ void tc_commit_pair(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
+}
+template <int KIND>
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    if (KIND == 0)
+        asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p; }"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    else if (KIND == 1)
+        asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p; }"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    else
+        asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p; }"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
 // 32 lanes x 32 consecutive fp32 columns: thread i receives row (lane base + i)
 __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -132,11 +183,12 @@ struct GemmParams {
 };
 enum { KIND_F16 = 0, KIND_I8 = 1, KIND_F8 = 2 };
 
-template <int BN>
+template <int BN, int CG>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
 {
-    constexpr int kStages = TileCfg<BN>::kStages, kStageBytes = TileCfg<BN>::kStageBytes, kTmemCols = TileCfg<BN>::kTmemCols;
+    using Cfg = TileCfg<BN, CG>;
+    constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes, kTmemCols = Cfg::kTmemCols;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], tfull_bar[2], tempty_bar[2];
     __shared__ uint32_t tmem_base_slot;
@@ -147,9 +199,12 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+    const int rank = CG == 2 ? (int)cluster_ctarank() : 0;            // 0 = leader of the pair
+    const int unit = (int)blockIdx.x / CG, n_units = (int)gridDim.x / CG;  // a unit (CTA or pair) owns whole tiles
+    const int tiles_m = (p.M + BM * CG - 1) / (BM * CG), tiles_n = (p.N + BN - 1) / BN;
     const int n_tiles = tiles_m * tiles_n;
-    const int kblocks = (p.K + p.bk - 1) / p.bk;
+    constexpr int KA = Cfg::KA;
+    const int kblocks = (p.K + p.bk * KA - 1) / (p.bk * KA);  // a k-block is one stage: KA atoms of K
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -158,18 +213,24 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&tfull_bar[b], 1);
-            mbar_init(&tempty_bar[b], 4);
+            mbar_init(&tempty_bar[b], 4 * CG);  // the epilogue warps of every CTA of the unit release the leader
         }
         err = 0;
         red[0] = red[1] = red[2] = red[3] = 0.0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // the MMA warp owns the tensor-memory allocation
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (CG == 2) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
-    __syncthreads();
+    if (CG == 2) cluster_sync();  // the peer's barriers are initialised before anything signals them
+    else __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&tmem_base_slot);
 
@@ -177,18 +238,33 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             int it = 0;
-            for (int tile = blockIdx.x; tile < n_tiles && !err; tile += gridDim.x) {
-                const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;  // m fastest: co-running tiles share a B tile
+            for (int tile = unit; tile < n_tiles && !err; tile += n_units) {
+                // m fastest: co-running tiles share a B tile.  This CTA's rows of A and of B inside the unit's tile:
+                const int m0 = (tile % tiles_m) * BM * CG + rank * BM, n0 = (tile / tiles_m) * BN + rank * Cfg::kBRows;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % kStages;
                     if (!mbar_wait(&empty_bar[s], ((it / kStages) & 1) ^ 1, perr)) break;
-                    mbar_expect_tx(&full_bar[s], kStageBytes);
                     unsigned char *st = smem + (size_t)s * kStageBytes;
-                    tma_load_2d(st, &map_a, kb * p.bk, m0, &full_bar[s]);
-                    tma_load_2d(st + kABytes, &map_b, kb * p.bk, n0, &full_bar[s]);
+                    // stage layout: KA atoms of A (16 KB each), then KA atoms of B
+                    if (CG == 2) {  // both CTAs' bytes are counted on the leader's barrier
+                        if (rank == 0) mbar_expect_tx(&full_bar[s], 2 * kStageBytes);
+                        const uint32_t leader_bar = mapa_u32(smem_u32(&full_bar[s]), 0);
+#pragma unroll
+                        for (int a = 0; a < KA; ++a) {
+                            tma_load_2d_pair(st + a * kABytes, &map_a, (kb * KA + a) * p.bk, m0, leader_bar);
+                            tma_load_2d_pair(st + KA * kABytes + a * Cfg::kBBytes, &map_b, (kb * KA + a) * p.bk, n0, leader_bar);
+                        }
+                    } else {
+                        mbar_expect_tx(&full_bar[s], kStageBytes);
+#pragma unroll
+                        for (int a = 0; a < KA; ++a) {
+                            tma_load_2d(st + a * kABytes, &map_a, (kb * KA + a) * p.bk, m0, &full_bar[s]);
+                            tma_load_2d(st + KA * kABytes + a * Cfg::kBBytes, &map_b, (kb * KA + a) * p.bk, n0, &full_bar[s]);
+                        }
+                    }
                 }
             }
-            if (err) {  // let copies that are still in flight land before the shared memory is given back
+            if (err && rank == 0) {  // let copies that are still in flight land before the shared memory is given back
                 for (int s = 0; s < kStages; ++s) {
                     const long long t0 = clock64();
                     while (!mbar_try_wait(&full_bar[s], 0) && !mbar_try_wait(&full_bar[s], 1) && clock64() - t0 < kWaitCycles) {}
@@ -197,9 +273,9 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             int it = 0, local = 0;
-            for (int tile = blockIdx.x; tile < n_tiles && !err; tile += gridDim.x, ++local) {
+            for (int tile = unit; tile < n_tiles && !err; tile += n_units, ++local) {
                 const int buf = local & 1;
                 if (!mbar_wait(&tempty_bar[buf], ((local >> 1) & 1) ^ 1, perr)) break;
                 tc_fence_after();
@@ -208,20 +284,31 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % kStages;
                     if (!mbar_wait(&full_bar[s], (it / kStages) & 1, perr)) { ok = false; break; }
-                    tc_fence_after();
+                    // (no tcgen05 fence here: the mbarrier orders the TMA data for the MMAs, and a fence would make
+                    //  this thread drain the MMAs of the previous k-block before issuing the next ones)
                     const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
-                    const uint64_t a_desc = smem_desc_k_major_sw128(sa), b_desc = smem_desc_k_major_sw128(sa + kABytes);
 #pragma unroll
-                    for (int k = 0; k < kRowBytes / 32; ++k) {  // one MMA consumes 32 bytes of K (16 x 16-bit or 32 x 8-bit)
-                        const uint64_t ad = a_desc + (uint64_t)(2 * k), bd = b_desc + (uint64_t)(2 * k);
-                        if (p.kind == KIND_F16) tc_mma_f16(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-                        else if (p.kind == KIND_I8) tc_mma_i8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-                        else tc_mma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                    for (int k = 0; k < KA * (kRowBytes / 32); ++k) {  // one MMA consumes 32 bytes of K (16 x 16-bit or 32 x 8-bit)
+                        const int atom = k / (kRowBytes / 32), kk = k % (kRowBytes / 32);
+                        const uint64_t ad = smem_desc_k_major_sw128(sa + atom * kABytes) + (uint64_t)(2 * kk);
+                        const uint64_t bd = smem_desc_k_major_sw128(sa + KA * kABytes + atom * Cfg::kBBytes) + (uint64_t)(2 * kk);
+                        if (CG == 2) {
+                            if (p.kind == KIND_F16) tc_mma_pair<0>(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                            else if (p.kind == KIND_I8) tc_mma_pair<1>(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                            else tc_mma_pair<2>(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                        } else {
+                            if (p.kind == KIND_F16) tc_mma_f16(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                            else if (p.kind == KIND_I8) tc_mma_i8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                            else tc_mma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                        }
                     }
-                    tc_commit(&empty_bar[s]);  // the stage is free once these MMAs have read it
+                    // the stage is free (in every CTA of the unit) once these MMAs have read it
+                    if (CG == 2) tc_commit_pair(&empty_bar[s]);
+                    else tc_commit(&empty_bar[s]);
                 }
                 if (!ok) break;
-                tc_commit(&tfull_bar[buf]);    // accumulator complete
+                if (CG == 2) tc_commit_pair(&tfull_bar[buf]);  // accumulator complete
+                else tc_commit(&tfull_bar[buf]);
             }
         }
     } else {
@@ -230,9 +317,9 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const float alpha = *p.alpha;
         double dsum = 0.0;
         int local = 0;
-        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++local) {
+        for (int tile = unit; tile < n_tiles; tile += n_units, ++local) {
             const int buf = local & 1;
-            const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;  // m fastest: co-running tiles share a B tile
+            const int m0 = (tile % tiles_m) * BM * CG + rank * BM, n0 = (tile / tiles_m) * BN;
             if (!mbar_wait(&tfull_bar[buf], (local >> 1) & 1, perr)) break;
             tc_fence_after();
             const int row = m0 + q * 32 + lane;
@@ -310,21 +397,26 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             dsum += (double)fsum;
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tempty_bar[buf]);
+            if (lane == 0) {
+                if (CG == 2 && rank != 0) mbar_arrive_cluster(mapa_u32(smem_u32(&tempty_bar[buf]), 0));
+                else mbar_arrive(&tempty_bar[buf]);
+            }
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
         if (lane == 0) red[q] = dsum;
     }
     tc_fence_before();
-    __syncthreads();
+    if (CG == 2) cluster_sync();  // no CTA leaves while its peer may still touch its shared or tensor memory
+    else __syncthreads();
     if (threadIdx.x == 0) {
         p.partials[blockIdx.x] = (red[0] + red[1]) + (red[2] + red[3]);
         if (err) atomicOr(p.status, MOFQ_STATUS_TIMEOUT);
     }
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        if (CG == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 #undef err
 }
@@ -475,16 +567,22 @@ int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, lon
              int op, int mode, float *Y, const float *alpha, const float *col_scale, double *partials, int32_t *status,
              int *grid_out, cudaStream_t st)
 {
-    // tile width: waves x relative tile cost (operand bytes per tile: 32 KB vs 48 KB per k-block)
+    // tile shape: waves x relative tile cost.  Operand bytes per CTA and k-block: 32 KB for a 128x128 tile, 48 KB for
+    // 128x256, and 32 KB per CTA for a CTA pair sharing a 256x256 tile (cost per 128x128 of output: 1, 0.75, 0.5).
     const int nsm = sm_count();
     const long long mt = (a_rows + BM - 1) / BM;
     const long long t128 = mt * ((b_rows + 127) / 128), t256 = mt * ((b_rows + 255) / 256);
+    const long long tpair = ((a_rows + 2 * BM - 1) / (2 * BM)) * ((b_rows + 255) / 256);
+    const int npair = std::max(1, nsm / 2);
     const double c128 = (double)((t128 + nsm - 1) / nsm) * 1.0, c256 = (double)((t256 + nsm - 1) / nsm) * 1.5;
-    const int bn = c256 < c128 ? 256 : 128;
+    const double cpair = (double)((tpair + npair - 1) / npair) * 1.0;
+    const bool force_single = getenv("MOFQ_GEMM_SINGLE_CTA") != nullptr;
+    const int cg = (!force_single && cpair < std::min(c128, c256)) ? 2 : 1;
+    const int bn = cg == 2 ? 256 : (c256 < c128 ? 256 : 128);
     CUtensorMap map_a, map_b;
     const int elem = op >= kOp8 ? kElemU8 : op;
     if (int rc = make_map(&map_a, a, elem, a_rows, K, a_ld, BM)) return rc;
-    if (int rc = make_map(&map_b, b, elem, b_rows, K, b_ld, bn)) return rc;
+    if (int rc = make_map(&map_b, b, elem, b_rows, K, b_ld, bn / cg)) return rc;
     GemmParams p{};
     p.M = (int)a_rows;
     p.N = (int)b_rows;
@@ -505,19 +603,36 @@ int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, lon
         p.kind = KIND_F16; cfmt = 1u; abfmt = op == MOFQ_F16 ? 0u : 1u /* f16 : bf16 */;
     }
     p.bk = op >= kOp8 ? kRowBytes : kRowBytes / 2;
-    p.idesc = (cfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-    const int tiles = (int)(((a_rows + BM - 1) / BM) * ((b_rows + bn - 1) / bn));
-    const int grid = std::min(tiles, std::min(sm_count(), kMaxGemmCtas));
+    p.idesc = (cfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((BM * cg) >> 4) << 24);
+    const int tiles = cg == 2 ? (int)tpair : (int)(((a_rows + BM - 1) / BM) * ((b_rows + bn - 1) / bn));
+    const int grid = cg * std::min(tiles, std::min(nsm, kMaxGemmCtas) / cg);
     const size_t smem = (size_t)kRingBytes + 1024;
     auto launch = [&](auto kernel) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
             (void)cudaGetLastError();
             return MOFQ_ERR_CUDA;
         }
-        kernel<<<grid, kGemmThreads, smem, st>>>(map_a, map_b, p);
-        return cudaGetLastError() == cudaSuccess ? MOFQ_OK : MOFQ_ERR_CUDA;
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3((unsigned)grid);
+        lc.blockDim = dim3(kGemmThreads);
+        lc.dynamicSmemBytes = smem;
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cg;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        if (cudaLaunchKernelEx(&lc, kernel, map_a, map_b, p) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MOFQ_ERR_CUDA;
+        }
+        return MOFQ_OK;
     };
-    if (int rc = bn == 256 ? launch(gemm_err_kernel<256>) : launch(gemm_err_kernel<128>)) return rc;
+    if (int rc = cg == 2 ? launch(gemm_err_kernel<256, 2>)
+                         : (bn == 256 ? launch(gemm_err_kernel<256, 1>) : launch(gemm_err_kernel<128, 1>)))
+        return rc;
     *grid_out = grid;
     return MOFQ_OK;
 }
