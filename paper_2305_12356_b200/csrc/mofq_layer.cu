@@ -21,6 +21,7 @@
 
 #include <algorithm>
 #include <cstdlib>
+#include <type_traits>
 
 #include "mofq_internal.h"
 
@@ -273,43 +274,57 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
+        // The tensor pipe takes an MMA only when it can start it, so whatever else this thread does between MMAs is
+        // a bubble: the loop is kept to a barrier wait, KA*4 MMAs whose descriptors are one 64-bit add away, a commit.
         if (lane == 0 && rank == 0) {
-            int it = 0, local = 0;
-            for (int tile = unit; tile < n_tiles && !err; tile += n_units, ++local) {
-                const int buf = local & 1;
-                if (!mbar_wait(&tempty_bar[buf], ((local >> 1) & 1) ^ 1, perr)) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                bool ok = true;
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    if (!mbar_wait(&full_bar[s], (it / kStages) & 1, perr)) { ok = false; break; }
-                    // (no tcgen05 fence here: the mbarrier orders the TMA data for the MMAs, and a fence would make
-                    //  this thread drain the MMAs of the previous k-block before issuing the next ones)
-                    const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
+            const uint32_t idesc = p.idesc;
+            const uint64_t a_desc0 = smem_desc_k_major_sw128(smem_u32(smem));
+            const uint64_t b_desc0 = smem_desc_k_major_sw128(smem_u32(smem + KA * kABytes));
+            auto run = [&](auto kind_tag) {
+                constexpr int KIND = decltype(kind_tag)::value;
+                int s = 0, local = 0;
+                uint32_t ph = 0;
+                uint64_t a_desc = a_desc0, b_desc = b_desc0;  // descriptors of the current stage (address field in 16-byte units)
+                for (int tile = unit; tile < n_tiles && !err; tile += n_units, ++local) {
+                    const int buf = local & 1;
+                    if (!mbar_wait(&tempty_bar[buf], ((local >> 1) & 1) ^ 1, perr)) return;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                    uint32_t acc = 0;
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        // (no tcgen05 fence here: the mbarrier orders the TMA data for the MMAs)
+                        if (!mbar_wait(&full_bar[s], ph, perr)) return;
 #pragma unroll
-                    for (int k = 0; k < KA * (kRowBytes / 32); ++k) {  // one MMA consumes 32 bytes of K (16 x 16-bit or 32 x 8-bit)
-                        const int atom = k / (kRowBytes / 32), kk = k % (kRowBytes / 32);
-                        const uint64_t ad = smem_desc_k_major_sw128(sa + atom * kABytes) + (uint64_t)(2 * kk);
-                        const uint64_t bd = smem_desc_k_major_sw128(sa + KA * kABytes + atom * Cfg::kBBytes) + (uint64_t)(2 * kk);
-                        if (CG == 2) {
-                            if (p.kind == KIND_F16) tc_mma_pair<0>(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-                            else if (p.kind == KIND_I8) tc_mma_pair<1>(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-                            else tc_mma_pair<2>(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                        for (int k = 0; k < KA * (kRowBytes / 32); ++k) {  // one MMA consumes 32 bytes of K
+                            constexpr int per = kRowBytes / 32;
+                            const uint64_t ad = a_desc + (uint64_t)((k / per) * (kABytes >> 4) + 2 * (k % per));
+                            const uint64_t bd = b_desc + (uint64_t)((k / per) * (Cfg::kBBytes >> 4) + 2 * (k % per));
+                            if (CG == 2) tc_mma_pair<KIND>(d_tmem, ad, bd, idesc, acc);
+                            else if (KIND == KIND_F16) tc_mma_f16(d_tmem, ad, bd, idesc, acc);
+                            else if (KIND == KIND_I8) tc_mma_i8(d_tmem, ad, bd, idesc, acc);
+                            else tc_mma_f8(d_tmem, ad, bd, idesc, acc);
+                            acc = 1;
+                        }
+                        // the stage is free (in every CTA of the unit) once these MMAs have read it
+                        if (CG == 2) tc_commit_pair(&empty_bar[s]);
+                        else tc_commit(&empty_bar[s]);
+                        if (++s == kStages) {
+                            s = 0;
+                            ph ^= 1u;
+                            a_desc = a_desc0;
+                            b_desc = b_desc0;
                         } else {
-                            if (p.kind == KIND_F16) tc_mma_f16(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-                            else if (p.kind == KIND_I8) tc_mma_i8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
-                            else tc_mma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                            a_desc += (uint64_t)(kStageBytes >> 4);
+                            b_desc += (uint64_t)(kStageBytes >> 4);
                         }
                     }
-                    // the stage is free (in every CTA of the unit) once these MMAs have read it
-                    if (CG == 2) tc_commit_pair(&empty_bar[s]);
-                    else tc_commit(&empty_bar[s]);
+                    if (CG == 2) tc_commit_pair(&tfull_bar[buf]);  // accumulator complete
+                    else tc_commit(&tfull_bar[buf]);
                 }
-                if (!ok) break;
-                if (CG == 2) tc_commit_pair(&tfull_bar[buf]);  // accumulator complete
-                else tc_commit(&tfull_bar[buf]);
-            }
+            };
+            if (p.kind == KIND_F16) run(std::integral_constant<int, KIND_F16>());
+            else if (p.kind == KIND_I8) run(std::integral_constant<int, KIND_I8>());
+            else run(std::integral_constant<int, KIND_F8>());
         }
     } else {
         // ---------------- epilogue: warps 2..5 read the lane quarter (warp % 4) of the accumulator ----------------
