@@ -149,6 +149,22 @@ int mofq_tensor_error(const mofq_tensor *x, const int32_t *formats, int n, int g
                       float *mse_out, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * mofq_absmax_update - running abs-max over calibration batches: *absmax_inout = max(*absmax_inout, max |x|)
+ * (Section 3.2, dynamic tensor analysis: the calibration process keeps the largest value seen over several batches to
+ * determine the scaling factor).  absmax_inout: device float, initialise it to 0 before the first batch.
+ */
+int mofq_absmax_update(const mofq_tensor *x, float *absmax_inout, void *stream);
+
+/*
+ * mofq_tensor_error_scaled - tensor MSE of n candidates under CALLER-SUPPLIED per-tensor scales, e.g. calibration scales
+ * applied to an unseen activation batch (Section 3.2, dynamic tensor analysis).  scales_in: device, n floats, one scale
+ * per candidate in the caller's order (typically calibration abs-max / format maximum); inv = RN32(1/scale); values
+ * beyond the grid saturate.  mse_out: device, n floats.  workspace as for mofq_tensor_error.
+ */
+int mofq_tensor_error_scaled(const mofq_tensor *x, const int32_t *formats, int n, const float *scales_in, float *mse_out,
+                             void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * mofq_layer_output_error - error of the layer output Y = X W^T when its inputs are quantised
  * (Section 3.2 layer analysis; Algorithm 1 `compute_error` with the layer output metric).
  * is_w_only: Yq = X dq(W)^T; otherwise Yq = dq(X) dq(W)^T with the same format for both tensors.

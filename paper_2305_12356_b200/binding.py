@@ -73,6 +73,10 @@ def lib():
                                                 vp, vp, vp]
         L.mofq_noalloc_scratch_bytes.restype = sz
         L.mofq_noalloc_scratch_bytes.argtypes = []
+        L.mofq_absmax_update.restype = C.c_int
+        L.mofq_absmax_update.argtypes = [C.POINTER(MofqTensor), vp, vp]
+        L.mofq_tensor_error_scaled.restype = C.c_int
+        L.mofq_tensor_error_scaled.argtypes = [C.POINTER(MofqTensor), C.POINTER(C.c_int32), C.c_int, vp, vp, vp, sz, vp]
         L.mofq_diag_fp_round.restype = C.c_int
         L.mofq_diag_fp_round.argtypes = [C.c_int, vp, vp, C.c_int64, vp]
         L.mofq_layer_output_error.restype = C.c_int
@@ -239,6 +243,27 @@ def tensor_error_noalloc(x, formats, gran, gran2=None, group=0, mse_out=None, st
     _check(L.mofq_tensor_error_noalloc(C.byref(d), fm, n, _gran(gran), g2, group, mse_out.data_ptr(),
                                        status_out.data_ptr(), _stream(x.device)))
     return mse_out, status_out
+
+
+def absmax_update(x, absmax):
+    """mofq_absmax_update: absmax (1-element float32 CUDA tensor) <- max(absmax, max|x|)."""
+    d = tensor_desc(x)
+    _check(lib().mofq_absmax_update(C.byref(d), absmax.data_ptr(), _stream(x.device)))
+    return absmax
+
+
+def tensor_error_scaled(x, formats, scales, workspace=None):
+    """mofq_tensor_error_scaled: MSE of each candidate under the given per-tensor scales (float32 CUDA tensor [n])."""
+    L = lib()
+    d = tensor_desc(x)
+    n = len(formats)
+    fm = (C.c_int32 * n)(*[_fmt(f) for f in formats])
+    sc = scales.contiguous().float()
+    assert sc.numel() == n and sc.is_cuda
+    out = torch.empty(n, dtype=torch.float32, device=x.device)
+    ws = workspace if workspace is not None else _workspace(L.mofq_tensor_workspace_bytes(C.byref(d)), x.device)
+    _check(L.mofq_tensor_error_scaled(C.byref(d), fm, n, sc.data_ptr(), out.data_ptr(), ws.data_ptr(), ws.numel(), _stream(x.device)))
+    return out, ws[:4].view(torch.int32)
 
 
 def diag_fp_round(fmt, t):

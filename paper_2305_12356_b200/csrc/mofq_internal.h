@@ -90,6 +90,8 @@ int sm_count();
 // kernels' host launchers (mofq_kq.cu)
 int launch_score(const ScoreJob &job, cudaStream_t st);
 int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st);
+int launch_absmax_update(const mofq_tensor &x, float *absmax_inout, cudaStream_t st);
+int launch_score_supplied(const ScoreJob &job, const float *scales, cudaStream_t st);
 int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in,
                 void *codes_out, float *scales_out, void *dequant_out, void *values_out, int values_dtype,
                 WsHeader *hdr, cudaStream_t st, int format_id = -1 /* mofq_format of f: enables the fused code kernel */);

@@ -457,6 +457,94 @@ kq_score_uniform(const uint16_t *__restrict__ x, long long rows, int chunks_per_
     block_finish<NC>(dacc, status, hdr, partials, fin, red);
 }
 
+// ---- caller-supplied per-tensor scales (calibration, Section 3.2 dynamic tensor analysis): saturating scorer -------
+// scales[i] belongs to the caller's candidate i; inv = RN32(1/scale); out-of-range values clip to the grid ends.
+template <int DT, int NI, int NFP>
+__global__ void __launch_bounds__(256)
+kq_score_supplied(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, CandSet cs,
+                  const float *__restrict__ scales, WsHeader *hdr, double *partials, Finalize fin)
+{
+    constexpr int NC = NI + NFP;
+    __shared__ double red[33 * NC];
+    float s[NC], inv[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+        s[j] = 1.0f;
+        for (int i = fin.n_cand - 1; i >= 0; --i)
+            if (fin.perm[i] == j) s[j] = scales[i];
+        inv[j] = __fdiv_rn(1.0f, s[j]);
+    }
+    double dacc[NC];
+    float acc[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+        dacc[j] = 0.0;
+        acc[j] = 0.0f;
+    }
+    int status = 0, n = 0;
+    const long long total = rows * chunks_per_row;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / chunks_per_row;
+        const int c = (int)(i - r * chunks_per_row);
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c);
+        if (mag16_nonfinite<DT>(fold16(absmax_chunk(v, 0)))) status |= MOFQ_STATUS_NONFINITE_INPUT;
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float xv[2];
+            unpack2<DT>(w[k], xv[0], xv[1]);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                if (NI) {
+                    const float t = fminf(fmaxf(__fmul_rn(xv[h], inv[0]), -1024.0f), 1024.0f);
+                    float q = __fsub_rn(__fadd_rn(t, kMagic), kMagic);
+                    q = fminf(fmaxf(q, -cs.int_q - 1.0f), cs.int_q);
+                    const float e = __fmaf_rn(-q, s[0], xv[h]);
+                    acc[0] = __fmaf_rn(e, e, acc[0]);
+                }
+#pragma unroll
+                for (int f = 0; f < NFP; ++f) {
+                    const float a = fabsf(xv[h]);
+                    const float t = fminf(__fmul_rn(a, inv[NI + f]), 2.0f * cs.fp_q[f]);
+                    const float q = fminf(fp_grid_round(t, cs.fp_eminb[f], cs.fp_kadd[f]), cs.fp_q[f]);
+                    const float e = __fmaf_rn(-q, s[NI + f], a);
+                    acc[NI + f] = __fmaf_rn(e, e, acc[NI + f]);
+                }
+            }
+        }
+        if (++n == 16) {
+#pragma unroll
+            for (int j = 0; j < NC; ++j) {
+                dacc[j] += (double)acc[j];
+                acc[j] = 0.0f;
+            }
+            n = 0;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < NC; ++j) dacc[j] += (double)acc[j];
+    block_finish<NC>(dacc, status, hdr, partials, fin, red);
+}
+
+// running abs-max over calibration batches: *absmax_inout = max(*absmax_inout, max |x|) (non-negative floats order like uints)
+template <int DT>
+__global__ void __launch_bounds__(256)
+kq_absmax_update(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, float *absmax_inout)
+{
+    uint32_t m = 0;
+    const long long total = rows * chunks_per_row;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / chunks_per_row;
+        const int c = (int)(i - r * chunks_per_row);
+        m = absmax_chunk(__ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c), m);
+    }
+    uint32_t m16 = fold16(m);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) m16 = max(m16, __shfl_xor_sync(0xffffffffu, m16, o));
+    if ((threadIdx.x & 31) == 0 && m16)
+        atomicMax(reinterpret_cast<uint32_t *>(absmax_inout), __float_as_uint(mag16_to_float<DT>(m16)));
+}
+
 // ---- emit kernel: codes / scales / dequantised values for ONE format ---------------------------------------
 // One row per block.  GRAN selects where the scale of a 16-byte chunk comes from.
 __device__ __forceinline__ uint32_t fp_code_from_mag(float r, const FmtDesc &f)
@@ -781,6 +869,36 @@ int sm_count()
         cached = n;
     }
     return cached;
+}
+
+int launch_absmax_update(const mofq_tensor &x, float *absmax_inout, cudaStream_t st)
+{
+    if (x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+    const uint16_t *xp = static_cast<const uint16_t *>(x.data);
+    const long long total = x.rows * (x.cols / 8);
+    const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
+    if (x.dtype == MOFQ_F16)
+        kq_absmax_update<0><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, absmax_inout);
+    else
+        kq_absmax_update<1><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, absmax_inout);
+    MOFQ_CUDA_OK(cudaGetLastError());
+    return MOFQ_OK;
+}
+
+// tensor error of every candidate under caller-supplied per-tensor scales (job.gran is ignored)
+int launch_score_supplied(const ScoreJob &job, const float *scales, cudaStream_t st)
+{
+    const mofq_tensor &x = job.x;
+    if (x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+    const uint16_t *xp = static_cast<const uint16_t *>(x.data);
+    const long long total = x.rows * (x.cols / 8);
+    const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
+    return dispatch_cands(x.dtype, job.cs.n_int, job.cs.n_fp, [&](auto DT, auto NI, auto NFP) {
+        kq_score_supplied<DT(), NI(), NFP()><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, job.cs, scales, job.hdr,
+                                                                    job.partials, job.fin);
+        MOFQ_CUDA_OK(cudaGetLastError());
+        return MOFQ_OK;
+    });
 }
 
 // abs-max of the whole tensor into hdr->absmax_bits (the caller has cleared that word)

@@ -310,3 +310,47 @@ def test_hardware_fp_rounding_matches_oracle(orc, dev, name):
     want = np.array([tab[orc.encode_fp_arith(fmt, v)] for v in t])
     np.testing.assert_array_equal(got.astype(np.float64), want)
     np.testing.assert_array_equal(np.signbit(got), np.signbit(t))               # the sign survives rounding to zero
+
+
+# ---- calibration scales applied to unseen batches (Section 3.2, dynamic tensor analysis) --------------------------------------
+def test_calibration_scales_and_saturation_match_oracle(orc, dev):
+    n_in, T = 1024, 256
+    batches = []
+    for b in range(5):
+        x = torch.empty((T, n_in), dtype=torch.bfloat16, device=dev)
+        inputs.device_activation(x, 61, b, n_ch=6, ch_gain=50.0 if b < 4 else 120.0)   # the unseen batch has larger outliers
+        batches.append(x)
+    cal = torch.zeros(1, dtype=torch.float32, device=dev)
+    for x in batches[:4]:
+        mofq.absmax_update(x, cal)
+    want_cal = max(float(host(x).abs().max()) for x in batches[:4])
+    assert float(cal.item()) == want_cal                                         # the largest value over the calibration batches
+    names = ["INT8", "FP8_E4M3", "FP8_E5M2"]
+    scales = torch.tensor([np.float32(want_cal) / np.float32(orc.format_max(getattr(orc, n))) for n in names], dtype=torch.float32, device=dev)
+    for x in (batches[1], batches[4]):                                           # a calibration batch and the unseen, clipping batch
+        got, st = mofq.tensor_error_scaled(x, names, scales)
+        want = [orc.quantize(host(x), getattr(orc, n), orc.PER_TENSOR, scales_in=[float(s)])["sse"] / x.numel()
+                for n, s in zip(names, scales.cpu())]
+        assert int(st.item()) == 0
+        assert rel_err(got.cpu().numpy(), want).max() < MSE_RTOL, (got, want)
+    # the paper's observation: with calibration scales FP8 has the lower error on activations with outliers
+    assert got[1].item() < got[0].item()
+    # candidate order is the caller's
+    got2, _ = mofq.tensor_error_scaled(batches[4], names[::-1], scales.flip(0))
+    assert torch.equal(got2.flip(0), got)
+
+
+@pytest.mark.parametrize("names", [["INT4", "FP4_E2M1"], ["FP4_E2M1_IEEE", "INT4", "FP4_E2M1"], ["FP8_E4M3"], ["INT8"]])
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_supplied_scales_small_and_ragged(orc, dev, names, dtype):
+    x = torch.empty((37, 1000), dtype=dtype, device=dev)                        # ragged: 37000 elements
+    inputs.device_weight(x, "gauss_outlier", 62, 0)
+    amax = float(host(x).abs().max())
+    for shrink in (1.0, 0.37, 2.5):                                              # exact, clipping, and wasteful scales
+        sc = torch.tensor([np.float32(amax * shrink) / np.float32(orc.format_max(getattr(orc, n))) for n in names],
+                          dtype=torch.float32, device=dev)
+        got, st = mofq.tensor_error_scaled(x, names, sc)
+        want = [orc.quantize(host(x), getattr(orc, n), orc.PER_TENSOR, scales_in=[float(s)])["sse"] / x.numel()
+                for n, s in zip(names, sc.cpu())]
+        assert int(st.item()) == 0
+        assert rel_err(got.cpu().numpy(), want).max() < MSE_RTOL, (names, shrink, got, want)
