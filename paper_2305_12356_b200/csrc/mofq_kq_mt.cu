@@ -8,7 +8,7 @@
 // candidate from the same registers.  Per (layer, CTA, warp) partial sums go to the workspace; a
 // second small kernel adds them in a fixed order and applies Algorithm 1's comparison.
 //
-// Arithmetic per element, on magnitudes a = |x| (every grid is symmetric):
+// Arithmetic per element a = x (signs kept; every grid is symmetric and both roundings are sign-symmetric):
 //   INT : r = RNE(a*inv) through fma(a, inv, 1.5*2^23) - 1.5*2^23.  The fused multiply-add rounds
 //         the exact product once instead of twice; the two can differ only where a*inv sits within
 //         one binary32 ulp of a tie, and at a tie both neighbours have the same error, so the
@@ -30,7 +30,14 @@
 namespace mofq {
 namespace {
 
-constexpr int kStages = 2;
+#ifndef MOFQ_MT_STAGES
+#define MOFQ_MT_STAGES 2
+#endif
+#ifndef MOFQ_MT_CTAS_PER_SM
+#define MOFQ_MT_CTAS_PER_SM 3
+#endif
+constexpr int kStages = MOFQ_MT_STAGES;
+constexpr int kCtasPerSm = MOFQ_MT_CTAS_PER_SM;   // kStages * kTileBytes * kCtasPerSm must fit one SM's shared memory
 constexpr int kTileBytes = 32768;
 constexpr int kConsumerWarps = 4;
 constexpr int kConsumers = kConsumerWarps * 32;
@@ -65,6 +72,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         }
     }
     return true;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
 }
 __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
 {
@@ -107,6 +120,9 @@ kq_score_mt(const MtParams p)
     __shared__ int err;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // tiles start on a 1 KB boundary of the shared window, so that a group's chunk addresses can be formed by XOR
+    const uint32_t smem_base = (smem_u32(smem) + 1023u) & ~1023u;
+    unsigned char *const smem_al = smem + (smem_base - smem_u32(smem));
     const long long t_begin = (long long)blockIdx.x * p.tiles_per_cta;
     const long long t_end = min(t_begin + p.tiles_per_cta, p.total_tiles);
     if (threadIdx.x == 0) {
@@ -142,7 +158,7 @@ kq_score_mt(const MtParams p)
                 const long long ng = min((long long)gpt, L.n_groups - g0);
                 const uint32_t bytes = (uint32_t)(ng * p.group * 2);
                 mbar_expect_tx(&full_bar[s], bytes);
-                bulk_load(smem + (size_t)s * kTileBytes, reinterpret_cast<const unsigned char *>(L.x) + ((size_t)(t - L.tile_begin) << (tile_elems_shift + 1)), bytes, &full_bar[s]);
+                bulk_load(smem_al + (size_t)s * kTileBytes, reinterpret_cast<const unsigned char *>(L.x) + ((size_t)(t - L.tile_begin) << (tile_elems_shift + 1)), bytes, &full_bar[s]);
             }
             if (err) {
                 // give copies already issued a bounded chance to land before the CTA's shared memory is released
@@ -195,16 +211,18 @@ kq_score_mt(const MtParams p)
         if (!mbar_wait(&full_bar[s], ph, &err)) break;
         const long long g0 = (t - L.tile_begin) * gpt;
         const int ng = (int)min((long long)gpt, L.n_groups - g0);
-        const uint4 *tile = reinterpret_cast<const uint4 *>(smem + (size_t)s * kTileBytes);
+        const uint32_t tile = smem_base + (uint32_t)s * kTileBytes;
         for (int g = threadIdx.x; g < ng; g += kConsumers) {
-            const uint4 *base = tile + g * cpg;
+            // chunk j of the group sits at a0 ^ (j << 4): the lane-dependent XOR spreads the lanes of a quarter-warp
+            // over all banks, and each address costs one logic instruction
+            const uint32_t a0 = tile + (uint32_t)g * (uint32_t)(cpg << 4) + (uint32_t)((g & (cpg - 1)) << 4);
             uint32_t m = 0;
             if (cpg == 16) {  // group of 128: fully unrolled
 #pragma unroll
-                for (int j = 0; j < 16; ++j) m = absmax_chunk<DT>(base[(j + g) & 15], m);
+                for (int j = 0; j < 16; ++j) m = absmax_chunk<DT>(lds128(a0 ^ (uint32_t)(j << 4)), m);
             } else {
 #pragma unroll 4
-                for (int j = 0; j < cpg; ++j) m = absmax_chunk<DT>(base[(j + g) & (cpg - 1)], m);
+                for (int j = 0; j < cpg; ++j) m = absmax_chunk<DT>(lds128(a0 ^ (uint32_t)(j << 4)), m);
             }
             const uint32_t m16 = fold16(m);
             if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
@@ -216,10 +234,10 @@ kq_score_mt(const MtParams p)
             scorer.begin(sc);
             if (cpg == 16) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) scorer.chunk(base[(j + g) & 15]);
+                for (int j = 0; j < 16; ++j) scorer.chunk(lds128(a0 ^ (uint32_t)(j << 4)));
             } else {
 #pragma unroll 4
-                for (int j = 0; j < cpg; ++j) scorer.chunk(base[(j + g) & (cpg - 1)]);
+                for (int j = 0; j < cpg; ++j) scorer.chunk(lds128(a0 ^ (uint32_t)(j << 4)));
             }
             scorer.end(dacc);
         }
@@ -301,7 +319,7 @@ template <int DT, int NI, int K0, int K1>
 int launch(const MtParams &p, int grid, cudaStream_t st)
 {
     auto kernel = kq_score_mt<DT, NI, K0, K1>;
-    const size_t smem = (size_t)kStages * kTileBytes;
+    const size_t smem = (size_t)kStages * kTileBytes + 1024;   // + slack to align the tiles
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
         (void)cudaGetLastError();
         return MOFQ_ERR_CUDA;
@@ -324,7 +342,7 @@ int dispatch(int ni, int k0, int k1, const MtParams &p, int grid, cudaStream_t s
 }
 
 size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
-int mt_grid() { return sm_count() * 3; }
+int mt_grid() { return sm_count() * kCtasPerSm; }
 
 }  // namespace
 
