@@ -184,6 +184,26 @@ int mofq_layer_output_error(const mofq_layer *L, const mofq_config *cfg, float *
 int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_config *cfg,
                         mofq_result *results_out, void *workspace, size_t workspace_bytes, void *stream);
 
+/* Where one layer's quantised weights go (device memory, caller-owned). */
+typedef struct mofq_packed {
+    void *codes;     /* rows*cols*bit_width/8 bytes, packed as by mofq_quantize_tensor */
+    float *scales;   /* one per row (per-channel), per group, or one (per-tensor)      */
+} mofq_packed;
+
+/*
+ * mofq_emit_selected - the last step of Algorithm 1: every layer keeps the quantisation of the format that
+ * won its selection.  The winner is read ON THE DEVICE from the layer's selection record, so this call can be
+ * enqueued right behind mofq_select_formats on the same stream with no host round trip in between.
+ *   results      device records written by mofq_select_formats with the same cfg (first granularity's record
+ *                of each layer when cfg->w_gran2 is given)
+ *   out          HOST array of n_layers destinations (device pointers inside); scales follow cfg->w_gran / w_group
+ *   formats_out  device, n_layers int32 (nullable): the mofq_format each layer was quantised to - the
+ *                per-layer format tag of the mixed-format model
+ *   workspace    device, at least 256 bytes; its first int32 holds the OR of the layers' status bits afterwards
+ */
+int mofq_emit_selected(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const mofq_result *results,
+                       const mofq_packed *out, int32_t *formats_out, void *workspace, size_t workspace_bytes, void *stream);
+
 /*
  * mofq_select_formats_host - the same selection for a model whose tensors live in HOST memory
  * (pinned memory recommended).  Layer data pointers are host pointers and the tensors are dense

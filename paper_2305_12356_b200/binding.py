@@ -73,6 +73,8 @@ def lib():
                                                 vp, vp, vp]
         L.mofq_noalloc_scratch_bytes.restype = sz
         L.mofq_noalloc_scratch_bytes.argtypes = []
+        L.mofq_emit_selected.restype = C.c_int
+        L.mofq_emit_selected.argtypes = [vp, C.c_int, C.POINTER(MofqConfig), vp, vp, vp, vp, sz, vp]
         L.mofq_absmax_update.restype = C.c_int
         L.mofq_absmax_update.argtypes = [C.POINTER(MofqTensor), vp, vp]
         L.mofq_tensor_error_scaled.restype = C.c_int
@@ -315,6 +317,37 @@ def select_formats(layers, cfg, workspace=None, results=None, parse=True):
     if not parse:
         return res
     return _parse_results(bytes(res.cpu().numpy()), n_rec, cfg.n_candidates)
+
+
+class MofqPacked(C.Structure):
+    _fields_ = [("codes", C.c_void_p), ("scales", C.c_void_p)]
+
+
+def emit_selected(layers, cfg, results):
+    """mofq_emit_selected: quantise every layer's W to the format its selection record names (read on the device).
+
+    `results` is the raw device byte tensor of select_formats(..., parse=False).  Returns (packed, formats, status):
+    packed = list of dict(codes uint8 tensor, scales float32 tensor) per layer, formats = int32 device tensor of
+    mofq_format tags, status = 1-element int32 device tensor.  Nothing synchronises.
+    """
+    L = lib()
+    prep = prepare_layers(layers)
+    dev = prep.device
+    n = len(prep)
+    out = (MofqPacked * n)()
+    packed = []
+    for i, layer in enumerate(prep.layers):
+        W = layer if torch.is_tensor(layer) else layer[0]
+        rows, cols = W.shape
+        codes = torch.empty(rows * cols * cfg.bit_width // 8, dtype=torch.uint8, device=dev)
+        scales = torch.empty(n_scales(cfg.w_gran, rows, cols, cfg.w_group), dtype=torch.float32, device=dev)
+        out[i].codes, out[i].scales = codes.data_ptr(), scales.data_ptr()
+        packed.append(dict(codes=codes, scales=scales))
+    formats = torch.empty(n, dtype=torch.int32, device=dev)
+    ws = _workspace(256, dev)
+    _check(L.mofq_emit_selected(prep.array, n, C.byref(cfg), results.data_ptr(), C.cast(out, C.c_void_p), formats.data_ptr(),
+                                ws.data_ptr(), ws.numel(), _stream(dev)))
+    return packed, formats, ws[:4].view(torch.int32)
 
 
 def select_formats_host(layers, cfg, device, workspace=None):

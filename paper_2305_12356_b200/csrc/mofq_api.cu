@@ -337,6 +337,35 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
     return MOFQ_OK;
 }
 
+int mofq_emit_selected(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const mofq_result *results,
+                       const mofq_packed *out, int32_t *formats_out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!layers || n_layers <= 0 || !results || !out) return MOFQ_ERR_INVALID_ARG;
+    if (int rc = check_config(cfg)) return rc;
+    if (int rc = check_ws(workspace, workspace_bytes, sizeof(WsHeader))) return rc;
+    EmitSel sel{};
+    for (int c = 0; c < cfg->n_candidates; ++c) {
+        if (!describe_format(cfg->candidates[c], &sel.cand[c]) || sel.cand[c].bits != cfg->bit_width) return MOFQ_ERR_INVALID_ARG;
+        sel.format[c] = cfg->candidates[c];
+    }
+    for (int i = 0; i < n_layers; ++i) {
+        if (int rc = check_tensor(&layers[i].W)) return rc;
+        if (int rc = check_gran(cfg->w_gran, cfg->w_group, layers[i].W.cols)) return rc;
+        if (!out[i].codes || !out[i].scales) return MOFQ_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
+    const int n_sets = cfg->w_gran2 != MOFQ_GRAN_NONE ? 2 : 1;
+    for (int i = 0; i < n_layers; ++i) {  // Algorithm 1, last step: the layer keeps the quantisation of its best format
+        sel.res = results + (size_t)i * n_sets;
+        sel.tag_out = formats_out ? formats_out + i : nullptr;
+        if (int rc = launch_emit(layers[i].W, sel.cand[0], cfg->w_gran, cfg->w_group, nullptr, out[i].codes, out[i].scales, nullptr,
+                                 nullptr, MOFQ_F16, static_cast<WsHeader *>(workspace), st, -1, &sel))
+            return rc;
+    }
+    return MOFQ_OK;
+}
+
 int mofq_select_formats_host(const mofq_layer *layers, int n_layers, const mofq_config *cfg, mofq_result *results_host,
                              void *workspace, size_t workspace_bytes, void *stream)
 {

@@ -87,6 +87,15 @@ int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const
            const int *fp_formats, mofq_result *results, void *ws, cudaStream_t st);
 int sm_count();
 
+// Format of an emit launch picked ON THE DEVICE from a selection record (Algorithm 1's last step without a host
+// round trip): the kernel quantises with cand[res->chosen] and stores that candidate's mofq_format in *tag_out.
+struct EmitSel {
+    const mofq_result *res;   // nullptr: the launch uses the format passed by value
+    int32_t *tag_out;         // nullable
+    FmtDesc cand[MOFQ_MAX_CAND];
+    int32_t format[MOFQ_MAX_CAND];
+};
+
 // kernels' host launchers (mofq_kq.cu)
 int launch_score(const ScoreJob &job, cudaStream_t st);
 int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st);
@@ -94,7 +103,8 @@ int launch_absmax_update(const mofq_tensor &x, float *absmax_inout, cudaStream_t
 int launch_score_supplied(const ScoreJob &job, const float *scales, cudaStream_t st);
 int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in,
                 void *codes_out, float *scales_out, void *dequant_out, void *values_out, int values_dtype,
-                WsHeader *hdr, cudaStream_t st, int format_id = -1 /* mofq_format of f: enables the fused code kernel */);
+                WsHeader *hdr, cudaStream_t st, int format_id = -1 /* mofq_format of f: enables the fused code kernel */,
+                const EmitSel *sel = nullptr /* format chosen on the device; f then only fixes the code width */);
 int launch_emit_codes_uniform(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
                               WsHeader *hdr, cudaStream_t st);
 int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,

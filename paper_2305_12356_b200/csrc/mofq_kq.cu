@@ -565,9 +565,14 @@ template <int DT, int GRAN>
 __global__ void __launch_bounds__(kRowThreads)
 kq_emit(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, FmtDesc f, int group,
         const float *__restrict__ scales_in, unsigned char *codes_out, float *scales_out, uint16_t *dequant_out,
-        uint16_t *values_out, int values_dtype, WsHeader *hdr)
+        uint16_t *values_out, int values_dtype, WsHeader *hdr, const EmitSel sel)
 {
     __shared__ uint32_t mred[34];
+    if (sel.res) {  // the winner of the selection record decides the grid
+        const int c = min(max(sel.res->chosen, 0), MOFQ_MAX_CAND - 1);
+        f = sel.cand[c];
+        if (sel.tag_out && blockIdx.x == 0 && threadIdx.x == 0) *sel.tag_out = sel.format[c];
+    }
     const int chunks = cols >> 3;
     const int lanes_per_group = GRAN == MOFQ_PER_GROUP ? (group >> 3) : 1;  // power of two <= 32
     const int gpr = GRAN == MOFQ_PER_GROUP ? cols / group : 1;
@@ -1058,8 +1063,13 @@ int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void
 
 int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in, void *codes_out,
                 float *scales_out, void *dequant_out, void *values_out, int values_dtype, WsHeader *hdr, cudaStream_t st,
-                int format_id)
+                int format_id, const EmitSel *sel)
 {
+    EmitSel es{};
+    if (sel) {
+        es = *sel;
+        format_id = -1;  // the fused code kernel needs the format on the host
+    }
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
     const int nsm = sm_count();
     if (x.cols > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
@@ -1084,7 +1094,7 @@ int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, con
     if (x.dtype == DT_ && gran == G_) {                                                                                      \
         kq_emit<DT_, G_><<<grid, kRowThreads, 0, st>>>(xp, x.rows, (int)x.cols, x.ld, f, group, scales_in,                   \
                                                        (unsigned char *)codes_out, scales_out, (uint16_t *)dequant_out,      \
-                                                       (uint16_t *)values_out, values_dtype, hdr);                           \
+                                                       (uint16_t *)values_out, values_dtype, hdr, es);                       \
         MOFQ_CUDA_OK(cudaGetLastError());                                                                                    \
         return MOFQ_OK;                                                                                                      \
     }
