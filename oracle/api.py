@@ -58,6 +58,11 @@ def lib():
                                              C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, f64p, f64p]
         L.orc_select.restype = C.c_int
         L.orc_select.argtypes = [f64p, C.c_int]
+        L.orc_block_sse.restype = C.c_int
+        L.orc_block_sse.argtypes = [u16p, C.c_int, i64, i64, i64, C.c_int, C.c_int, C.c_int, f64p]
+        L.orc_select_blocks.restype = C.c_int
+        L.orc_select_blocks.argtypes = [u16p, C.c_int, i64, i64, i64, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int,
+                                        u8p, f64p, f64p]
         L.orc_num_threads.restype = C.c_int
         L.orc_num_threads.argtypes = []
         L.orc_crosscheck_fp.restype = C.c_int64
@@ -212,6 +217,31 @@ def layer_output_error(X, W, fmt, is_w_only, w_gran=PER_CHANNEL, w_group=0, a_gr
 def select(errors):
     e = np.ascontiguousarray(errors, dtype=np.float64)
     return lib().orc_select(_ptr(e, C.c_double), e.size)
+
+
+def block_sse(x, fmt, gran, group=0):
+    """Sum of squared errors of every scale block (row or group), each quantised with its own abs-max scale."""
+    bits, dt = as_bits(x)
+    rows, cols = bits.shape
+    out = np.empty(n_scales(gran, rows, cols, group), np.float64)
+    if lib().orc_block_sse(_ptr(bits, C.c_uint16), dt, rows, cols, cols, fmt, gran, group, _ptr(out, C.c_double)):
+        raise ValueError("oracle: bad argument")
+    return out
+
+
+def select_blocks(x, fmts, gran, group=0):
+    """Block-wise format selection.  Returns dict(choice uint8 [blocks], block_sse float64 [blocks, n], mixed_mse)."""
+    bits, dt = as_bits(x)
+    rows, cols = bits.shape
+    nb = n_scales(gran, rows, cols, group)
+    fm = (C.c_int * len(fmts))(*fmts)
+    choice = np.empty(nb, np.uint8)
+    sse = np.empty((nb, len(fmts)), np.float64)
+    mixed = C.c_double()
+    if lib().orc_select_blocks(_ptr(bits, C.c_uint16), dt, rows, cols, cols, fm, len(fmts), gran, group,
+                               _ptr(choice, C.c_uint8), _ptr(sse, C.c_double), C.byref(mixed)):
+        raise ValueError("oracle: bad argument")
+    return dict(choice=choice, block_sse=sse, mixed_mse=mixed.value)
 
 
 def crosscheck_fp(fmt, lo_bits, hi_bits, stride=1):

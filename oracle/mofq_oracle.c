@@ -17,7 +17,8 @@
  * Pins (tests/test_oracle_*.py): Table 3 of the paper for the FP4 code->value map, enumeration
  * counts and library decodes for FP8, hand-made tie grids, closed-form uniform-noise MSE,
  * exact-rational brute force on tiny tensors, identity-activation and exact-integer special
- * cases for the layer output error.  No function in this file is "parity unpinned".
+ * cases for the layer output error; block-wise selection against row/group slices scored as
+ * tensors of their own and a hand-worked two-row case.  No function in this file is "parity unpinned".
  *
  * OpenMP is used only over rows / output rows (independent work items).
  */
@@ -32,7 +33,8 @@
 /* ORC_MUTATION (default 0 = none) plants one deliberate mistake; it exists only so that a test can show that the
  * pins reject a wrong oracle.  1: FP ties away from zero  2: E4M3 top code treated as a value (max 480)
  * 3: scale uses Q+1  4: MSE divides by rows instead of rows*cols  5: layer output uses W^T indexing swapped
- * 6: selection uses <=  7: subnormals flushed (no gradual underflow)  8: INT ties away from zero */
+ * 6: selection uses <=  7: subnormals flushed (no gradual underflow)  8: INT ties away from zero
+ * 9: blocks numbered group-major instead of row-major */
 #ifndef ORC_MUTATION
 #define ORC_MUTATION 0
 #endif
@@ -455,6 +457,76 @@ int orc_select(const double *errors, int n)
         if (errors[i] < min_error) { min_error = errors[i]; best = i; }
 #endif
     return best;
+}
+
+/* ---- finer-than-layer selection (Section 7 names channel-wise / block-wise mixing of formats as the next step;
+ *      Section 3.2 already scores per channel) ------------------------------------------------------------------
+ * A "block" is one scale block: a row (per-channel scales) or a run of `group` elements of a row (group
+ * scales).  Each block is quantised with its own abs-max scale; sse_out[b] is the block's sum of squared errors
+ * in double.  Blocks are numbered like the scales: row-major, groups left to right.
+ */
+int orc_block_sse(const uint16_t *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                  int fmt, int gran, int group, double *sse_out)
+{
+    fmt_t f;
+    if (fmt_lookup(fmt, &f)) return -1;
+    if (gran == ORC_PER_GROUP && (group <= 0 || cols % group)) return -1;
+    int64_t width = gran == ORC_PER_GROUP ? group : cols;     /* elements per block within a row */
+    int64_t per_row = gran == ORC_PER_TENSOR ? 0 : cols / width;
+    if (gran == ORC_PER_TENSOR) {                               /* degenerate: the whole tensor is the one block */
+        return orc_quantize(x, dtype, rows, cols, ld, fmt, gran, group, NULL, NULL, NULL, NULL, sse_out);
+    }
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t b = 0; b < per_row; ++b) {
+            const uint16_t *blk = x + r * ld + b * width;
+            float amax = 0.0f;
+            for (int64_t c = 0; c < width; ++c) {
+                float a = fabsf(orc_load(blk + c, dtype));
+                if (a > amax || isnan(a)) amax = a;
+            }
+            float scale, inv;
+            orc_scale_from_absmax(fmt, amax, &scale, &inv);
+            double sse = 0.0;
+            for (int64_t c = 0; c < width; ++c) {
+                float xv = orc_load(blk + c, dtype);
+                float t = xv * inv;
+                int code = f.is_fp ? orc_encode_fp_arith(fmt, t, sign_bit16(blk[c])) : orc_encode_int(fmt, t);
+                double e = (double)xv - orc_decode(fmt, code) * (double)scale;
+                sse += e * e;
+            }
+#if ORC_MUTATION == 9
+            sse_out[b * rows + r] = sse;
+#else
+            sse_out[r * per_row + b] = sse;
+#endif
+        }
+    return 0;
+}
+
+/* Per block, Algorithm 1's rule applied to the block errors: the first candidate (caller's order) with the strictly
+ * smallest SSE.  choice_out[b] = index into fmts; mixed_mse_out = sum of the chosen SSEs / element count. */
+int orc_select_blocks(const uint16_t *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                      const int *fmts, int n_fmts, int gran, int group, uint8_t *choice_out, double *block_sse_out,
+                      double *mixed_mse_out)
+{
+    int64_t nb = n_scales(gran, rows, cols, group);
+    double *sse = (double *)malloc(sizeof(double) * (size_t)(nb * n_fmts));
+    int rc = 0;
+    for (int k = 0; k < n_fmts && !rc; ++k)
+        rc = orc_block_sse(x, dtype, rows, cols, ld, fmts[k], gran, group, sse + (int64_t)k * nb);
+    double total = 0.0;
+    for (int64_t b = 0; b < nb && !rc; ++b) {
+        double e[8];
+        for (int k = 0; k < n_fmts; ++k) e[k] = sse[(int64_t)k * nb + b];
+        int best = orc_select(e, n_fmts);
+        choice_out[b] = (uint8_t)best;
+        total += e[best];
+        if (block_sse_out)
+            for (int k = 0; k < n_fmts; ++k) block_sse_out[b * n_fmts + k] = e[k];
+    }
+    if (!rc) *mixed_mse_out = (rows > 0 && cols > 0) ? total / (double)(rows * cols) : 0.0;
+    free(sse);
+    return rc;
 }
 
 /* ---- cross-check helper: arithmetic vs table FP rounding over a range of binary32 patterns ----

@@ -18,6 +18,7 @@ MUTATIONS = {
     6: "tests/test_oracle_quantize.py::test_selection_strict_less_first_wins_ties",
     7: "tests/test_oracle_formats.py::test_all_midpoints_and_grid_points",
     8: "tests/test_oracle_formats.py::test_int_rounding_ties_to_even_and_clamp",
+    9: "tests/test_oracle_blocks.py::test_block_equals_the_slice_scored_as_its_own_tensor",
 }
 
 
