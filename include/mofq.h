@@ -149,6 +149,21 @@ int mofq_tensor_error(const mofq_tensor *x, const int32_t *formats, int n, int g
                       float *mse_out, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * mofq_select_blocks - format selection finer than a layer: one winner per scale block, i.e. per output channel
+ * (gran = MOFQ_PER_CHANNEL) or per group of `group` elements (MOFQ_PER_GROUP).  Section 7 names channel-wise and
+ * block-wise mixing of formats as the step after layer-wise selection; the rule applied to every block is
+ * Algorithm 1's (strictly smaller error, caller's candidate order), the error being the block's sum of squared
+ * errors under its own abs-max scale.
+ *   formats        n candidates of one bit-width, n <= 3
+ *   choice_out     device, one byte per block (row-major, groups left to right): index into formats - the format map
+ *   block_sse_out  device, blocks*n floats (nullable): every block's error per candidate, caller's order
+ *   mse_out        device, n + 1 floats: whole-tensor MSE of each candidate, then of the per-block mixture
+ *   workspace      as for mofq_tensor_error
+ */
+int mofq_select_blocks(const mofq_tensor *x, const int32_t *formats, int n, int gran, int group, uint8_t *choice_out,
+                       float *block_sse_out, float *mse_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * mofq_absmax_update - running abs-max over calibration batches: *absmax_inout = max(*absmax_inout, max |x|)
  * (Section 3.2, dynamic tensor analysis: the calibration process keeps the largest value seen over several batches to
  * determine the scaling factor).  absmax_inout: device float, initialise it to 0 before the first batch.

@@ -75,6 +75,8 @@ def lib():
         L.mofq_noalloc_scratch_bytes.argtypes = []
         L.mofq_emit_selected.restype = C.c_int
         L.mofq_emit_selected.argtypes = [vp, C.c_int, C.POINTER(MofqConfig), vp, vp, vp, vp, sz, vp]
+        L.mofq_select_blocks.restype = C.c_int
+        L.mofq_select_blocks.argtypes = [C.POINTER(MofqTensor), C.POINTER(C.c_int32), C.c_int, C.c_int, C.c_int, vp, vp, vp, vp, sz, vp]
         L.mofq_absmax_update.restype = C.c_int
         L.mofq_absmax_update.argtypes = [C.POINTER(MofqTensor), vp, vp]
         L.mofq_tensor_error_scaled.restype = C.c_int
@@ -245,6 +247,24 @@ def tensor_error_noalloc(x, formats, gran, gran2=None, group=0, mse_out=None, st
     _check(L.mofq_tensor_error_noalloc(C.byref(d), fm, n, _gran(gran), g2, group, mse_out.data_ptr(),
                                        status_out.data_ptr(), _stream(x.device)))
     return mse_out, status_out
+
+
+def select_blocks(x, formats, gran, group=0, want_block_sse=False, workspace=None):
+    """mofq_select_blocks.  Returns dict(choice uint8 [blocks], block_sse float32 [blocks, n] or None,
+    mse float32 [n + 1] (candidates, then the mixture), status int32 tensor); nothing synchronises."""
+    L = lib()
+    d = tensor_desc(x)
+    n = len(formats)
+    fm = (C.c_int32 * n)(*[_fmt(f) for f in formats])
+    rows, cols = x.shape
+    nb = n_scales(gran, rows, cols, group)
+    choice = torch.empty(nb, dtype=torch.uint8, device=x.device)
+    sse = torch.empty((nb, n), dtype=torch.float32, device=x.device) if want_block_sse else None
+    mse = torch.empty(n + 1, dtype=torch.float32, device=x.device)
+    ws = workspace if workspace is not None else _workspace(L.mofq_tensor_workspace_bytes(C.byref(d)), x.device)
+    _check(L.mofq_select_blocks(C.byref(d), fm, n, _gran(gran), group, choice.data_ptr(), sse.data_ptr() if sse is not None else None,
+                                mse.data_ptr(), ws.data_ptr(), ws.numel(), _stream(x.device)))
+    return dict(choice=choice, block_sse=sse, mse=mse, status=ws[:4].view(torch.int32))
 
 
 def absmax_update(x, absmax):

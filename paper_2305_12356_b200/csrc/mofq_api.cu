@@ -246,6 +246,40 @@ int mofq_tensor_error(const mofq_tensor *x, const int32_t *formats, int n, int g
     return score_layer_tensor(*x, &cfg, cs, perm, nc, fp_formats, nullptr, mse_out, workspace, st);
 }
 
+int mofq_select_blocks(const mofq_tensor *x, const int32_t *formats, int n, int gran, int group, uint8_t *choice_out,
+                       float *block_sse_out, float *mse_out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (int rc = check_tensor(x)) return rc;
+    if (!choice_out || !mse_out || !formats || n < 1 || n > MOFQ_MAX_CAND - 1) return MOFQ_ERR_INVALID_ARG;
+    if (gran != MOFQ_PER_CHANNEL && gran != MOFQ_PER_GROUP) return MOFQ_ERR_UNSUPPORTED;
+    if (int rc = check_gran(gran, group, x->cols)) return rc;
+    FmtDesc d0;
+    if (!describe_format(formats[0], &d0)) return MOFQ_ERR_INVALID_ARG;
+    CandSet cs;
+    int perm[MOFQ_MAX_CAND], nc, fp_formats[2];
+    if (int rc = build_candset(formats, n, d0.bits, &cs, perm, &nc, fp_formats)) return rc;
+    if (int rc = check_ws(workspace, workspace_bytes, mofq_tensor_workspace_bytes(x))) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
+    ScoreJob job{};
+    job.x = *x;
+    job.cs = cs;
+    job.gran = gran;
+    job.gran2 = MOFQ_GRAN_NONE;
+    job.group = group;
+    job.fp_formats[0] = fp_formats[0];
+    job.fp_formats[1] = fp_formats[1];
+    job.hdr = static_cast<WsHeader *>(workspace);
+    job.partials = reinterpret_cast<double *>(static_cast<char *>(workspace) + sizeof(WsHeader));
+    job.fin.mse_out = mse_out;
+    job.fin.n_cand = n;
+    job.fin.n_sets = 1;
+    job.fin.nc = nc;
+    std::memcpy(job.fin.perm, perm, sizeof(job.fin.perm));
+    job.fin.inv_n = 1.0 / ((double)x->rows * (double)x->cols);
+    return launch_select_blocks(job, choice_out, block_sse_out, st);
+}
+
 int mofq_absmax_update(const mofq_tensor *x, float *absmax_inout, void *stream)
 {
     if (int rc = check_tensor(x)) return rc;

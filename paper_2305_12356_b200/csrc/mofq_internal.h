@@ -101,6 +101,8 @@ int launch_score(const ScoreJob &job, cudaStream_t st);
 int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st);
 int launch_absmax_update(const mofq_tensor &x, float *absmax_inout, cudaStream_t st);
 int launch_score_supplied(const ScoreJob &job, const float *scales, cudaStream_t st);
+// one winner per scale block; job.fin.mse_out receives n_cand + 1 floats (candidates, then the mixture)
+int launch_select_blocks(const ScoreJob &job, uint8_t *choice, float *block_sse, cudaStream_t st);
 int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in,
                 void *codes_out, float *scales_out, void *dequant_out, void *values_out, int values_dtype,
                 WsHeader *hdr, cudaStream_t st, int format_id = -1 /* mofq_format of f: enables the fused code kernel */,

@@ -11,6 +11,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <cstring>
 #include <type_traits>
 
 #include "kq_math.cuh"
@@ -397,6 +398,107 @@ kq_score_rows(const uint16_t *__restrict__ x, long long rows, int cols, long lon
             for (int j = 0; j < NC; ++j) dacc[j] += GRP ? a_g[j] : a_c[j];
         }
         __syncthreads();
+    }
+    block_finish<NA>(dacc, status, hdr, partials, fin, red);
+}
+
+// ---- block-wise selection: one winner per scale block (row or group) ---------------------------------------
+// A team of T lanes (a quarter of the block's chunks when that is a power of two <= 32, else a whole warp) owns one
+// block at a time, up to four chunks per lane held in registers: abs-max by shuffles, scales, then every candidate's squared error from the same registers; lane 0
+// of the team applies Algorithm 1's rule (strictly smaller, caller's order) to the block's errors.  Accumulators:
+// [canonical slots][mixture].
+struct BlockSel {
+    uint8_t *choice;     // [blocks] index into the caller's candidate list
+    float *block_sse;    // nullable: [blocks][n_cand], caller's order
+    int n_cand;
+    int perm[MOFQ_MAX_CAND];
+};
+
+template <int DT, int NI, int K0, int K1>
+__global__ void __launch_bounds__(256)
+kq_select_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, int width, int team, RowQ rq,
+                 BlockSel bs, WsHeader *hdr, double *partials, Finalize fin)
+{
+    // unscaled accumulation: a block can be as small as 8 elements, where the scaled form's rounding of x * inv
+    // (relative to x, not to the error) would show in the block's own sum
+    using S = kqmath::Scorer<DT, NI, K0, K1, false>;
+    constexpr int NC = S::NC;
+    constexpr int NA = NC + 1;
+    __shared__ double red[33 * NA];
+    const int lane = threadIdx.x & 31;
+    const int tl = lane & (team - 1);                       // lane within the team
+    const int teams_per_warp = 32 / team;
+    const int cpb = width >> 3;                             // 16-byte chunks per block
+    const int per_row = cols / width;
+    const long long n_blocks = rows * per_row;
+    const long long warp_id = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const long long n_warps = (long long)gridDim.x * (blockDim.x >> 5);
+    constexpr int KPL = 4;                                  // chunks a lane can keep in registers
+    const bool one_pass = cpb <= KPL * team;                // the block is read once; else twice (second read from cache)
+    double dacc[NA];
+#pragma unroll
+    for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
+    int status = 0;
+
+    for (long long b0 = warp_id * teams_per_warp; b0 < n_blocks; b0 += n_warps * teams_per_warp) {
+        const long long b = b0 + lane / team;
+        const bool live = b < n_blocks;                     // whole teams are live or not; shuffles stay warp-wide
+        const long long r = live ? b / per_row : 0;
+        const uint4 *blk = reinterpret_cast<const uint4 *>(x + r * ld + (live ? (b - r * per_row) * width : 0));
+        uint4 v[KPL];
+        uint32_t m = 0;
+        if (one_pass) {
+#pragma unroll
+            for (int k = 0; k < KPL; ++k) {
+                const int q = tl + k * team;
+                v[k] = (live && q < cpb) ? __ldg(blk + q) : make_uint4(0, 0, 0, 0);
+                m = kqmath::absmax_chunk<DT>(v[k], m);
+            }
+        } else if (live) {
+            for (int q = tl; q < cpb; q += team) m = kqmath::absmax_chunk<DT>(__ldg(blk + q), m);
+        }
+        uint32_t m16 = kqmath::fold16(m);
+        for (int o = team >> 1; o; o >>= 1) m16 = max(m16, __shfl_xor_sync(0xffffffffu, m16, o));
+        if (kqmath::mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+        const float a = kqmath::mag16_to_float<DT>(m16);
+        kqmath::Sc<NC> sc;
+#pragma unroll
+        for (int j = 0; j < NC; ++j) kqmath::scale_pair(a, rq.q[j], sc.s[j], sc.inv[j], status);
+        S scorer;
+        scorer.begin(sc);
+        if (one_pass) {
+#pragma unroll
+            for (int k = 0; k < KPL; ++k) scorer.chunk(v[k]);   // zeros (idle slots) add nothing
+        } else if (live) {
+            for (int q = tl; q < cpb; q += team) scorer.chunk(__ldg(blk + q));
+        }
+        float e[NC];
+#pragma unroll
+        for (int j = 0; j < NC; ++j) {
+            float lo, hi;
+            kqmath::upk(scorer.acc2[j], lo, hi);
+            e[j] = lo + hi;
+            for (int o = team >> 1; o; o >>= 1) e[j] += __shfl_xor_sync(0xffffffffu, e[j], o);
+        }
+        if (live && tl == 0) {
+            float best = INFINITY;
+            int pick = 0;
+            for (int i = 0; i < bs.n_cand; ++i) {
+                float ei = e[0];
+#pragma unroll
+                for (int j = 1; j < NC; ++j)
+                    if (bs.perm[i] == j) ei = e[j];
+                if (bs.block_sse) bs.block_sse[b * bs.n_cand + i] = ei;
+                if (ei < best) {                            // strictly smaller: the first candidate keeps a tie
+                    best = ei;
+                    pick = i;
+                }
+            }
+            bs.choice[b] = (uint8_t)pick;
+#pragma unroll
+            for (int j = 0; j < NC; ++j) dacc[j] += (double)e[j];
+            dacc[NC] += (double)best;
+        }
     }
     block_finish<NA>(dacc, status, hdr, partials, fin, red);
 }
@@ -907,6 +1009,53 @@ int launch_score_supplied(const ScoreJob &job, const float *scales, cudaStream_t
 }
 
 // abs-max of the whole tensor into hdr->absmax_bits (the caller has cleared that word)
+int launch_select_blocks(const ScoreJob &job, uint8_t *choice, float *block_sse, cudaStream_t st)
+{
+    const mofq_tensor &x = job.x;
+    if (job.gran != MOFQ_PER_CHANNEL && job.gran != MOFQ_PER_GROUP) return MOFQ_ERR_UNSUPPORTED;
+    if (x.cols > 0x7fffffffLL || job.fin.n_cand + 1 > MOFQ_MAX_CAND) return MOFQ_ERR_UNSUPPORTED;
+    const int width = job.gran == MOFQ_PER_GROUP ? job.group : (int)x.cols;
+    const int cpb = width >> 3;
+    const int team = (cpb <= 128 && (cpb & (cpb - 1)) == 0) ? std::max(1, cpb / 4) : 32;
+    const long long n_blocks = x.rows * (x.cols / width);
+    const long long warps = (n_blocks + (32 / team) - 1) / (32 / team);
+    const int grid = (int)std::min<long long>((warps + 7) / 8, std::min<long long>((long long)sm_count() * 8, kMaxSlots));
+    RowQ rq{};
+    if (job.cs.n_int) rq.q[0] = job.cs.int_q;
+    for (int f = 0; f < job.cs.n_fp; ++f) rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
+    auto kind = [](int format) {
+        return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
+    };
+    const int k0 = job.cs.n_fp > 0 ? kind(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? kind(job.fp_formats[1]) : -1;
+    BlockSel bs{};
+    bs.choice = choice;
+    bs.block_sse = block_sse;
+    bs.n_cand = job.fin.n_cand;
+    std::memcpy(bs.perm, job.fin.perm, sizeof(bs.perm));
+    // the finalize step reports the candidates in the caller's order and then the mixture (accumulator nc)
+    Finalize fin = job.fin;
+    fin.perm[fin.n_cand] = fin.nc;
+    fin.n_cand += 1;
+    fin.nc += 1;
+    const uint16_t *xp = static_cast<const uint16_t *>(x.data);
+#define MOFQ_BLK(DT_, NI_, K0_, K1_)                                                                              \
+    if (x.dtype == DT_ && job.cs.n_int == NI_ && k0 == K0_ && k1 == K1_) {                                        \
+        kq_select_blocks<DT_, NI_, K0_, K1_><<<grid, 256, 0, st>>>(xp, x.rows, (int)x.cols, x.ld, width, team, rq, bs, job.hdr, \
+                                                                    job.partials, fin);                          \
+        MOFQ_CUDA_OK(cudaGetLastError());                                                                         \
+        return MOFQ_OK;                                                                                           \
+    }
+#define MOFQ_BLK_DT(DT_)                                                                                          \
+    MOFQ_BLK(DT_, 1, -1, -1) MOFQ_BLK(DT_, 0, 0, -1) MOFQ_BLK(DT_, 1, 0, -1) MOFQ_BLK(DT_, 0, 0, 0) MOFQ_BLK(DT_, 1, 0, 0) \
+    MOFQ_BLK(DT_, 0, 1, -1) MOFQ_BLK(DT_, 1, 1, -1) MOFQ_BLK(DT_, 0, 2, -1) MOFQ_BLK(DT_, 1, 2, -1)               \
+    MOFQ_BLK(DT_, 0, 1, 2) MOFQ_BLK(DT_, 1, 1, 2) MOFQ_BLK(DT_, 0, 2, 1) MOFQ_BLK(DT_, 1, 2, 1)
+    MOFQ_BLK_DT(0)
+    MOFQ_BLK_DT(1)
+#undef MOFQ_BLK_DT
+#undef MOFQ_BLK
+    return MOFQ_ERR_UNSUPPORTED;
+}
+
 int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st)
 {
     if (x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
