@@ -331,7 +331,7 @@ def main():
         launches_per_step = len(shapes) * (3 + 4 * F + 2) if layer_metric else (3 + (len(shapes) + 63) // 64 if grans == ("group",) else len(shapes))
         mt = grans == ("group",)
         dom_launches = 1 if mt else len(shapes)      # launches of the dominant kernel per step
-        roofline = {"bound": "hbm", "kernel": "kq_score_mt" if mt else "kq_score_rows", "achieved": fp16_bytes / (ms_per_step * 1e-3) / 1e9,
+        roofline = {"bound": "hbm", "kernel": "kq_score_mt" if mt else "kq_score_rows_stream", "achieved": fp16_bytes / (ms_per_step * 1e-3) / 1e9,
                     "peak": peak, "peak_source": f"of {which}", "unit": "GB/s",
                     "frac": fp16_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
                     "frac_of_nominal_8TBs": fp16_bytes / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,

@@ -15,6 +15,7 @@
 #include <type_traits>
 
 #include "kq_math.cuh"
+#include "kq_pipe.cuh"
 #include "mofq_internal.h"
 
 namespace mofq {
@@ -498,6 +499,167 @@ kq_select_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long 
 #pragma unroll
             for (int j = 0; j < NC; ++j) dacc[j] += (double)e[j];
             dacc[NC] += (double)best;
+        }
+    }
+    block_finish<NA>(dacc, status, hdr, partials, fin, red);
+}
+
+// ---- scoring kernel 2b: whole rows streamed through a shared-memory ring --------------------------------------
+// Per-channel scales (optionally group-128 scales from the same read) for rows that are a multiple of 128
+// elements.  A tile is `rows_per_tile` whole rows; one producer thread brings tiles in with bulk asynchronous
+// copies that complete on mbarriers (two stages), the consumer threads own 128-element segments of the tile.
+// Pass 1: segment abs-max -> shared-memory max per row; a named barrier over the consumers; pass 2: every segment
+// is scored against its row's scales (and its own group scales) from shared memory.  Chunk addresses are formed
+// by XOR, as in the multi-tensor kernel.  All waits are bounded; a consumer that gave up still meets the
+// barriers, so nobody is left waiting for it.
+constexpr int kRsStages = 2;
+constexpr int kRsMaxRows = 8;
+constexpr int kRsMaxTileBytes = 49152;
+constexpr int kRsMaxConsumers = 256;
+
+struct RsParams {
+    const uint16_t *x;
+    long long rows, ld, n_tiles, tiles_per_cta;
+    int cols, rows_per_tile, segs_per_row, consumers, stage_bytes, grp_first;
+    RowQ rq;
+};
+
+template <int DT, int NI, int K0, int K1, bool GRP>
+__global__ void __launch_bounds__(kRsMaxConsumers + 32)
+kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize fin)
+{
+    using namespace kqpipe;
+    using S = kqmath::Scorer<DT, NI, K0, K1, true>;      // scales are fixed over a segment: scaled accumulation
+    constexpr int NC = S::NC;
+    constexpr int NA = NC * (GRP ? 2 : 1);
+    extern __shared__ __align__(16) unsigned char smem[];   // aligned by hand below
+    __shared__ __align__(8) uint64_t full_bar[kRsStages], empty_bar[kRsStages];
+    __shared__ uint32_t rowmax[4][kRsMaxRows];
+    __shared__ int err;
+    __shared__ double red[33 * NA];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_cw = p.consumers >> 5;
+    const uint32_t smem_base = (smem_u32(smem) + 1023u) & ~1023u;
+    unsigned char *const smem_al = smem + (smem_base - smem_u32(smem));
+    if (tid == 0) {
+        for (int s = 0; s < kRsStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], n_cw);
+        }
+        err = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < 4 * kRsMaxRows) (&rowmax[0][0])[tid] = 0;
+    __syncthreads();
+    const long long t_begin = (long long)blockIdx.x * p.tiles_per_cta;
+    const long long t_end = min(t_begin + p.tiles_per_cta, p.n_tiles);
+    const uint32_t row_bytes = (uint32_t)p.cols * 2u;
+    double dacc[NA];
+#pragma unroll
+    for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
+    int status = 0;
+
+    if (warp == n_cw) {
+        // ---------------- producer ----------------
+        if (lane == 0) {
+            int it = 0;
+            for (long long t = t_begin; t < t_end; ++t, ++it) {
+                const int s = it % kRsStages;
+                const uint32_t ph = (uint32_t)(it / kRsStages) & 1u;
+                if (!mbar_wait(&empty_bar[s], ph ^ 1u, &err)) break;
+                const long long r0 = t * p.rows_per_tile;
+                const int nr = (int)min((long long)p.rows_per_tile, p.rows - r0);
+                mbar_expect_tx(&full_bar[s], (uint32_t)nr * row_bytes);
+                unsigned char *dst = smem_al + (size_t)s * p.stage_bytes;
+                if (p.ld == p.cols) {
+                    bulk_load(dst, p.x + r0 * p.ld, (uint32_t)nr * row_bytes, &full_bar[s]);
+                } else {
+                    for (int r = 0; r < nr; ++r) bulk_load(dst + (size_t)r * row_bytes, p.x + (r0 + r) * p.ld, row_bytes, &full_bar[s]);
+                }
+            }
+            if (err) {
+                // give copies already issued a bounded chance to land before the shared memory is released
+                for (int s = 0; s < kRsStages; ++s) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&full_bar[s], 0) && !mbar_try_wait(&full_bar[s], 1) && clock64() - t0 < kWaitCycles) {}
+                }
+                status |= MOFQ_STATUS_TIMEOUT;
+            }
+        }
+    } else {
+        // ---------------- consumers ----------------
+        int it = 0;
+        for (long long t = t_begin; t < t_end; ++t, ++it) {
+            const int s = it % kRsStages;
+            const uint32_t ph = (uint32_t)(it / kRsStages) & 1u;
+            const bool ok = mbar_wait(&full_bar[s], ph, &err);
+            const long long r0 = t * p.rows_per_tile;
+            const int nr = (int)min((long long)p.rows_per_tile, p.rows - r0);
+            const int nseg = ok ? nr * p.segs_per_row : 0;
+            const uint32_t tile = smem_base + (uint32_t)s * (uint32_t)p.stage_bytes;
+            uint32_t *rmax = rowmax[it & 3];
+            uint32_t a0[2], segmax[2];
+            int srow[2];
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {                // at most two segments per consumer (the host sizes the tile so)
+                const int sg = tid + k * p.consumers;
+                segmax[k] = 0;
+                srow[k] = 0;
+                a0[k] = 0;
+                if (sg < nseg) {
+                    srow[k] = sg / p.segs_per_row;
+                    a0[k] = tile + (uint32_t)srow[k] * row_bytes + (uint32_t)(sg - srow[k] * p.segs_per_row) * 256u + (uint32_t)((tid & 15) << 4);
+                    uint32_t m = 0;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) m = kqmath::absmax_chunk<DT>(lds128(a0[k] ^ (uint32_t)(j << 4)), m);
+                    segmax[k] = kqmath::fold16(m);
+                    atomicMax(&rmax[srow[k]], segmax[k]);
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(p.consumers) : "memory");
+            // the buffer two tiles ahead was last read two tiles ago: everyone has left it by now
+            if (tid < kRsMaxRows) rowmax[(it + 2) & 3][tid] = 0;
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int sg = tid + k * p.consumers;
+                if (sg < nseg) {
+                    const uint32_t rm = rmax[srow[k]];
+                    if (kqmath::mag16_nonfinite<DT>(rm)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+                    kqmath::Sc<NC> sc;
+                    S s_c, s_g;
+#pragma unroll
+                    for (int j = 0; j < NC; ++j) kqmath::scale_pair(kqmath::mag16_to_float<DT>(rm), p.rq.q[j], sc.s[j], sc.inv[j], status);
+                    s_c.begin(sc);
+                    if (GRP) {
+#pragma unroll
+                        for (int j = 0; j < NC; ++j) kqmath::scale_pair(kqmath::mag16_to_float<DT>(segmax[k]), p.rq.q[j], sc.s[j], sc.inv[j], status);
+                        s_g.begin(sc);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const uint4 v = lds128(a0[k] ^ (uint32_t)(j << 4));
+                        s_c.chunk(v);
+                        if (GRP) s_g.chunk(v);
+                    }
+                    double a_c[NC], a_g[NC];
+#pragma unroll
+                    for (int j = 0; j < NC; ++j) a_c[j] = a_g[j] = 0.0;
+                    s_c.end(a_c);
+                    if (GRP) {
+                        s_g.end(a_g);
+#pragma unroll
+                        for (int j = 0; j < NC; ++j) {
+                            dacc[j] += p.grp_first ? a_g[j] : a_c[j];
+                            dacc[NC + j] += p.grp_first ? a_c[j] : a_g[j];
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < NC; ++j) dacc[j] += a_c[j];
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[s]);
         }
     }
     block_finish<NA>(dacc, status, hdr, partials, fin, red);
@@ -1070,6 +1232,78 @@ int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st)
     return MOFQ_OK;
 }
 
+namespace {
+
+int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
+{
+    const mofq_tensor &x = job.x;
+    const int spr = (int)(x.cols / 128);
+    const int row_bytes = (int)x.cols * 2;
+    // tile shape: whole rows, at most two 128-element segments per consumer thread, consumers a multiple of 32;
+    // take the shape that keeps the most consumer lanes busy, then the one with more tiles in flight
+    int best_r = 0, best_t = 0;
+    double best_eff = 0.0;
+    for (int r = 1; r <= kRsMaxRows && (long long)r <= x.rows && r * row_bytes <= kRsMaxTileBytes; ++r) {
+        const int nseg = r * spr;
+        for (int rounds = 1; rounds <= 2; ++rounds) {
+            const int t = 32 * ((nseg + 32 * rounds - 1) / (32 * rounds));
+            if (t > kRsMaxConsumers) continue;
+            const double eff = (double)nseg / ((double)t * rounds) * (r * row_bytes <= 32768 ? 1.0 : 0.97);
+            if (eff > best_eff + 1e-9 || (eff > best_eff - 1e-9 && r * row_bytes <= 32768)) {   // ties: the larger tile up to 32 KB
+                best_eff = eff;
+                best_r = r;
+                best_t = t;
+            }
+        }
+    }
+    if (!best_r) return MOFQ_ERR_UNSUPPORTED;
+    RsParams p{};
+    p.x = static_cast<const uint16_t *>(x.data);
+    p.rows = x.rows;
+    p.ld = x.ld;
+    p.cols = (int)x.cols;
+    p.rows_per_tile = best_r;
+    p.segs_per_row = spr;
+    p.consumers = best_t;
+    p.stage_bytes = (best_r * row_bytes + 1023) & ~1023;
+    p.grp_first = (job.gran == MOFQ_PER_GROUP) ? 1 : 0;
+    if (job.cs.n_int) p.rq.q[0] = job.cs.int_q;
+    for (int f = 0; f < job.cs.n_fp; ++f) p.rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
+    p.n_tiles = (x.rows + best_r - 1) / best_r;
+    const size_t smem = (size_t)kRsStages * p.stage_bytes + 1024;
+    const int threads = best_t + 32;
+    auto kind = [](int format) {
+        return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
+    };
+    const int k0 = job.cs.n_fp > 0 ? kind(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? kind(job.fp_formats[1]) : -1;
+    auto launch = [&](auto kernel) {
+        if (int rc = set_smem(kernel, smem)) return rc;
+        const int occ = std::max(1, blocks_per_sm((const void *)kernel, threads, smem));
+        long long grid = std::min<long long>(p.n_tiles, std::min<long long>((long long)sm_count() * occ, kMaxSlots));
+        p.tiles_per_cta = (p.n_tiles + grid - 1) / grid;
+        grid = (p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
+        kernel<<<(int)grid, threads, smem, st>>>(p, job.hdr, job.partials, job.fin);
+        MOFQ_CUDA_OK(cudaGetLastError());
+        return MOFQ_OK;
+    };
+#define MOFQ_RS(DT_, NI_, K0_, K1_)                                                                     \
+    if (x.dtype == DT_ && job.cs.n_int == NI_ && k0 == K0_ && k1 == K1_) {                              \
+        if (has_grp) return launch(kq_score_rows_stream<DT_, NI_, K0_, K1_, true>);                     \
+        return launch(kq_score_rows_stream<DT_, NI_, K0_, K1_, false>);                                 \
+    }
+#define MOFQ_RS_DT(DT_)                                                                                          \
+    MOFQ_RS(DT_, 1, -1, -1) MOFQ_RS(DT_, 0, 0, -1) MOFQ_RS(DT_, 1, 0, -1) MOFQ_RS(DT_, 0, 0, 0) MOFQ_RS(DT_, 1, 0, 0) \
+    MOFQ_RS(DT_, 0, 1, -1) MOFQ_RS(DT_, 1, 1, -1) MOFQ_RS(DT_, 0, 2, -1) MOFQ_RS(DT_, 1, 2, -1)                         \
+    MOFQ_RS(DT_, 0, 1, 2) MOFQ_RS(DT_, 1, 1, 2) MOFQ_RS(DT_, 0, 2, 1) MOFQ_RS(DT_, 1, 2, 1)
+    MOFQ_RS_DT(0)
+    MOFQ_RS_DT(1)
+#undef MOFQ_RS_DT
+#undef MOFQ_RS
+    return MOFQ_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
 int launch_score(const ScoreJob &job, cudaStream_t st)
 {
     const mofq_tensor &x = job.x;
@@ -1117,6 +1351,8 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
 
     // row kernel: per-channel, per-group on a strided tensor, or both from one read
     if (x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
+    if (has_ch && x.cols % 128 == 0 && x.cols * 2 <= kRsMaxTileBytes && (!has_grp || job.group == 128))
+        return launch_score_rows_stream(job, has_grp, st);
     const int chunks = (int)(x.cols / 8);
     const int gpr = has_grp ? (int)(x.cols / job.group) : 0;
     const size_t smem = (size_t)x.cols * 2 + (((size_t)chunks * 2 + 15) & ~(size_t)15) + (size_t)gpr * 8 * 3 + 16;

@@ -354,3 +354,19 @@ def test_supplied_scales_small_and_ragged(orc, dev, names, dtype):
                 for n, s in zip(names, sc.cpu())]
         assert int(st.item()) == 0
         assert rel_err(got.cpu().numpy(), want).max() < MSE_RTOL, (names, shrink, got, want)
+
+
+# ---- streamed-row scoring kernel: tile shapes, ragged last tile, strided rows, widest row ------------------------------------
+@pytest.mark.parametrize("rows,cols,ld", [(13, 128, 128), (37, 4096, 4096), (29, 6656, 6656 + 256), (5, 22016, 22016), (1, 24576, 24576),
+                                          (1100, 256, 256)])
+def test_streamed_rows_shapes(orc, dev, rows, cols, ld):
+    full = _weights(dev, rows, ld, seed=41, layer=rows % 7)
+    x = full[:, :cols]
+    names = ["INT4", "FP4_E2M1"]
+    got, st = mofq.tensor_error(x, names, "channel")
+    want = _oracle_mse(orc, host(x).contiguous(), names, "channel", 0)
+    assert int(st.item()) == 0
+    assert rel_err(got.cpu().numpy(), want).max() < MSE_RTOL
+    got2, _ = mofq.tensor_error(x, names, "group", gran2="channel", group=128)
+    want2 = _oracle_mse(orc, host(x).contiguous(), names, "group", 128) + want
+    assert rel_err(got2.cpu().numpy().reshape(-1), want2).max() < MSE_RTOL
