@@ -270,6 +270,14 @@ size_t mofq_noalloc_scratch_bytes(void);
  */
 int mofq_diag_fp_round(int format, const float *t, float *out, int64_t n, void *stream);
 
+/*
+ * mofq_diag_scale_pair - diagnostic: scale = RN32(a / Q) and inv = RN32(Q / a) (Section 3.2: abs-max scaling; a = 0
+ * gives 1, 1) as the multi-tensor scoring kernel computes them for binary16 tensors, i.e. without the general
+ * division routine.  Valid for abs-max values a binary16 tensor can have (0 or 2^-24 ... 65504); a test compares
+ * every such value with two correctly rounded divisions.  absmax, scale_out, inv_out: device, n floats.
+ */
+int mofq_diag_scale_pair(int format, const float *absmax, float *scale_out, float *inv_out, int64_t n, void *stream);
+
 /* Workspace sizes in bytes (host-side arithmetic only). */
 size_t mofq_tensor_workspace_bytes(const mofq_tensor *x);
 size_t mofq_workspace_bytes(const mofq_layer *layers, int n_layers, const mofq_config *cfg);

@@ -81,6 +81,8 @@ def lib():
         L.mofq_absmax_update.argtypes = [C.POINTER(MofqTensor), vp, vp]
         L.mofq_tensor_error_scaled.restype = C.c_int
         L.mofq_tensor_error_scaled.argtypes = [C.POINTER(MofqTensor), C.POINTER(C.c_int32), C.c_int, vp, vp, vp, sz, vp]
+        L.mofq_diag_scale_pair.restype = C.c_int
+        L.mofq_diag_scale_pair.argtypes = [C.c_int, vp, vp, vp, C.c_int64, vp]
         L.mofq_diag_fp_round.restype = C.c_int
         L.mofq_diag_fp_round.argtypes = [C.c_int, vp, vp, C.c_int64, vp]
         L.mofq_layer_output_error.restype = C.c_int
@@ -286,6 +288,14 @@ def tensor_error_scaled(x, formats, scales, workspace=None):
     ws = workspace if workspace is not None else _workspace(L.mofq_tensor_workspace_bytes(C.byref(d)), x.device)
     _check(L.mofq_tensor_error_scaled(C.byref(d), fm, n, sc.data_ptr(), out.data_ptr(), ws.data_ptr(), ws.numel(), _stream(x.device)))
     return out, ws[:4].view(torch.int32)
+
+
+def diag_scale_pair(fmt, absmax):
+    """mofq_diag_scale_pair: (scale, inv) of the multi-tensor kernel for a float32 CUDA tensor of abs-max values."""
+    a = absmax.contiguous().float()
+    s, inv = torch.empty_like(a), torch.empty_like(a)
+    _check(lib().mofq_diag_scale_pair(_fmt(fmt), a.data_ptr(), s.data_ptr(), inv.data_ptr(), a.numel(), _stream(a.device)))
+    return s, inv
 
 
 def diag_fp_round(fmt, t):

@@ -17,7 +17,21 @@ __global__ void diag_round(const float *__restrict__ t, float *__restrict__ out,
     if (i + 1 < n) out[i + 1] = copysignf(r.y, b);
 }
 
+__global__ void diag_scale_pair(const float *__restrict__ a, float Q, float rQ, float *__restrict__ s, float *__restrict__ inv, long long n)
+{
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) mofq::kqmath::scale_pair_fast(a[i], Q, rQ, s[i], inv[i]);
+}
+
 }  // namespace
+
+extern "C" int mofq_diag_scale_pair(int format, const float *absmax, float *scale_out, float *inv_out, int64_t n, void *stream)
+{
+    mofq::FmtDesc d;
+    if (!absmax || !scale_out || !inv_out || n <= 0 || !mofq::describe_format(format, &d)) return MOFQ_ERR_INVALID_ARG;
+    diag_scale_pair<<<(int)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(absmax, d.Q, 1.0f / d.Q, scale_out, inv_out, n);
+    return cudaGetLastError() == cudaSuccess ? MOFQ_OK : MOFQ_ERR_CUDA;
+}
 
 extern "C" int mofq_diag_fp_round(int format, const float *t, float *out, int64_t n, void *stream)
 {

@@ -302,7 +302,8 @@ kq_score_groups(const uint16_t *__restrict__ x, long long n_groups, int group, C
 constexpr int kRowThreads = 256;
 
 struct RowQ {
-    float q[3];  // abs-max target per canonical slot
+    float q[3];   // abs-max target per canonical slot
+    float rq[3];  // RN32(1 / q), for the division-free scale computation
 };
 
 template <int DT, int NI, int K0, int K1, bool CH, bool GRP>
@@ -628,11 +629,17 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
                     kqmath::Sc<NC> sc;
                     S s_c, s_g;
 #pragma unroll
-                    for (int j = 0; j < NC; ++j) kqmath::scale_pair(kqmath::mag16_to_float<DT>(rm), p.rq.q[j], sc.s[j], sc.inv[j], status);
+                    for (int j = 0; j < NC; ++j) {
+                        if (DT == MOFQ_F16) kqmath::scale_pair_fast(kqmath::mag16_to_float<DT>(rm), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
+                        else kqmath::scale_pair(kqmath::mag16_to_float<DT>(rm), p.rq.q[j], sc.s[j], sc.inv[j], status);
+                    }
                     s_c.begin(sc);
                     if (GRP) {
 #pragma unroll
-                        for (int j = 0; j < NC; ++j) kqmath::scale_pair(kqmath::mag16_to_float<DT>(segmax[k]), p.rq.q[j], sc.s[j], sc.inv[j], status);
+                        for (int j = 0; j < NC; ++j) {
+                            if (DT == MOFQ_F16) kqmath::scale_pair_fast(kqmath::mag16_to_float<DT>(segmax[k]), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
+                            else kqmath::scale_pair(kqmath::mag16_to_float<DT>(segmax[k]), p.rq.q[j], sc.s[j], sc.inv[j], status);
+                        }
                         s_g.begin(sc);
                     }
 #pragma unroll
@@ -1269,6 +1276,7 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
     p.grp_first = (job.gran == MOFQ_PER_GROUP) ? 1 : 0;
     if (job.cs.n_int) p.rq.q[0] = job.cs.int_q;
     for (int f = 0; f < job.cs.n_fp; ++f) p.rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
+    for (int j = 0; j < 3; ++j) p.rq.rq[j] = p.rq.q[j] > 0.0f ? 1.0f / p.rq.q[j] : 0.0f;
     p.n_tiles = (x.rows + best_r - 1) / best_r;
     const size_t smem = (size_t)kRsStages * p.stage_bytes + 1024;
     const int threads = best_t + 32;

@@ -54,6 +54,7 @@ struct MtParams {
     long long total_tiles, tiles_per_cta;
     int group;
     float q[3];          // abs-max target per canonical slot
+    float rq[3];         // RN32(1 / q)
     double *partials;    // [slot][kMaxAcc]
     int32_t *status;     // [layer]
     int32_t *timeout;    // one word: set if a bounded wait expired
@@ -190,7 +191,11 @@ kq_score_mt(const MtParams p)
             const float a = mag16_to_float<DT>(m16);
             Sc<NC> sc;
 #pragma unroll
-            for (int j = 0; j < NC; ++j) scale_pair(a, p.q[j], sc.s[j], sc.inv[j], status);
+            for (int j = 0; j < NC; ++j) {
+                // binary16 abs-max values cannot overflow the reciprocal: the short division-free sequence is exact there
+                if (DT == MOFQ_F16) scale_pair_fast(a, p.q[j], p.rq[j], sc.s[j], sc.inv[j]);
+                else scale_pair(a, p.q[j], sc.s[j], sc.inv[j], status);
+            }
             S scorer;
             scorer.begin(sc);
             if (cpg == 16) {
@@ -374,6 +379,7 @@ int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const
     p.group = cfg->w_group;
     if (cs.n_int) p.q[0] = cs.int_q;
     for (int f = 0; f < cs.n_fp; ++f) p.q[cs.n_int + f] = cs.fp_q[f];
+    for (int j = 0; j < 3; ++j) p.rq[j] = p.q[j] > 0.0f ? 1.0f / p.q[j] : 0.0f;
     p.partials = d_partials;
     p.status = d_status;
     p.timeout = d_status + n_layers;

@@ -370,3 +370,20 @@ def test_streamed_rows_shapes(orc, dev, rows, cols, ld):
     got2, _ = mofq.tensor_error(x, names, "group", gran2="channel", group=128)
     want2 = _oracle_mse(orc, host(x).contiguous(), names, "group", 128) + want
     assert rel_err(got2.cpu().numpy().reshape(-1), want2).max() < MSE_RTOL
+
+
+@pytest.mark.parametrize("name", FMT4 + FMT8)
+def test_fast_scale_pair_is_correctly_rounded_for_every_binary16_magnitude(orc, dev, name):
+    from paper_2305_12356_b200.binding import diag_scale_pair
+    bits = np.arange(0x7C00, dtype=np.uint16)                                    # 0, every subnormal and normal magnitude
+    a = bits.view(np.float16).astype(np.float32)
+    s, inv = diag_scale_pair(name, torch.from_numpy(a).to(dev))
+    Q = np.float32(orc.format_max(getattr(orc, name)))
+    with np.errstate(divide="ignore"):
+        want_s = np.where(a == 0, np.float32(1), a / Q).astype(np.float32)       # numpy float32 division is correctly rounded
+        want_i = np.where(a == 0, np.float32(1), Q / a).astype(np.float32)
+    np.testing.assert_array_equal(s.cpu().numpy().view(np.uint32), want_s.view(np.uint32))
+    np.testing.assert_array_equal(inv.cpu().numpy().view(np.uint32), want_i.view(np.uint32))
+    for k in (0, 1, 2, 1000, 0x3C00, 0x7BFF):                                    # and the oracle's own routine on a few
+        so, io = orc.scale_from_absmax(getattr(orc, name), a[k])
+        assert so == want_s[k] and io == want_i[k]
