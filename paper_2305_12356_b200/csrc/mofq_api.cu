@@ -124,6 +124,14 @@ int score_layer_tensor(const mofq_tensor &W, const mofq_config *cfg, const CandS
         if (int rc = check_gran(cfg->w_gran2, cfg->w_group, W.cols)) return rc;
         if (cfg->w_gran2 == cfg->w_gran) return MOFQ_ERR_INVALID_ARG;
     }
+    // a large dense tensor with group scales goes through the multi-tensor kernel as a list of one layer (its three
+    // small helper launches cost more than they save below a few tens of MB)
+    mofq_layer one{};
+    one.W = W;
+    if (cfg->metric == MOFQ_TENSOR_MSE && W.rows * W.cols >= (32LL << 20) && mt_applicable(&one, 1, cfg) &&
+        sizeof(WsHeader) + mt_ws_bytes(1) <= score_ws_bytes())
+        return mt_run(&one, 1, cfg, cs, perm, nc, fp_formats, res, static_cast<char *>(ws) + sizeof(WsHeader), st, mse_out,
+                      res ? nullptr : &static_cast<WsHeader *>(ws)->status);   // a record carries its own status
     ScoreJob job{};
     job.x = W;
     job.cs = cs;

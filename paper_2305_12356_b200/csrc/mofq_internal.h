@@ -84,7 +84,8 @@ struct MtLayer {
 bool mt_applicable(const mofq_layer *layers, int n_layers, const mofq_config *cfg);
 size_t mt_ws_bytes(int n_layers);
 int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
-           const int *fp_formats, mofq_result *results, void *ws, cudaStream_t st);
+           const int *fp_formats, mofq_result *results /* nullable */, void *ws, cudaStream_t st,
+           float *mse_out = nullptr /* [layer][candidate] */, int32_t *status_out = nullptr /* OR of the layers' status bits */);
 int sm_count();
 
 // Format of an emit launch picked ON THE DEVICE from a selection record (Algorithm 1's last step without a host

@@ -256,7 +256,10 @@ kq_mt_finalize(const MtLayer *layers, const double *partials, int32_t *status, c
     }
     r.rel_margin = best > 0.0 ? (float)((second - best) / best) : INFINITY;
     r.reserved = 0;
-    results[blockIdx.x] = r;
+    if (results) results[blockIdx.x] = r;
+    if (fin.mse_out)
+        for (int i = 0; i < fin.n_cand; ++i) fin.mse_out[(size_t)blockIdx.x * fin.n_cand + i] = r.error[i];
+    if (fin.status_out && r.status) atomicOr(fin.status_out, r.status);
 }
 
 // The work table travels to the device as kernel arguments, 64 entries per launch: fully stream-ordered,
@@ -330,7 +333,7 @@ size_t mt_ws_bytes(int n_layers)
 }
 
 int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
-           const int *fp_formats, mofq_result *results, void *ws, cudaStream_t st)
+           const int *fp_formats, mofq_result *results, void *ws, cudaStream_t st, float *mse_out, int32_t *status_out)
 {
     const int grid = mt_grid();
     const int gpt = (kTileBytes / 2) / cfg->w_group;
@@ -392,6 +395,8 @@ int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const
     fin.n_cand = cfg->n_candidates;
     fin.n_sets = 1;
     fin.nc = nc;
+    fin.mse_out = mse_out;
+    fin.status_out = status_out;
     for (int i = 0; i < MOFQ_MAX_CAND; ++i) fin.perm[i] = perm[i];
     kq_mt_finalize<<<n_layers, 128, 0, st>>>(d_table, d_partials, d_status, d_status + n_layers, fin, results);
     if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;

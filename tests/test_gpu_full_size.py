@@ -100,3 +100,19 @@ def test_layer_output_full_size_one_hot_activations(orc, dev, name, layer_index)
     assert rec["chosen"] == orc.select(want_mse)
     del w, x
     torch.cuda.empty_cache()
+
+
+def test_large_single_tensor_group_scales_takes_the_streaming_route(orc, dev):
+    """A dense tensor of >= 32 Mi elements with group scales is scored by the multi-tensor kernel as a one-layer list."""
+    w = torch.empty((11008, 4096), dtype=torch.float16, device=dev)       # 45 M elements, a LLaMA-7B gate projection
+    inputs.device_weight(w, "student_t", 5, 1)
+    names = ["FP4_E2M1", "INT4"]
+    got, st = mofq.tensor_error(w, names, "group", group=128)
+    want = [orc.tensor_mse(host(w), getattr(orc, n), orc.PER_GROUP, 128) for n in names]
+    assert int(st.item()) == 0
+    assert rel_err(got.cpu().numpy(), want).max() < MSE_RTOL
+    again, _ = mofq.tensor_error(w, names, "group", group=128)
+    assert torch.equal(got, again)                                         # fixed summation order
+    w[7000, 123] = float("inf")
+    _, st = mofq.tensor_error(w, names, "group", group=128)
+    assert int(st.item()) & mofq.binding.STATUS_NONFINITE_INPUT
