@@ -508,12 +508,14 @@ kq_select_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long 
 // ---- scoring kernel 2b: whole rows streamed through a shared-memory ring --------------------------------------
 // Per-channel scales (optionally group-128 scales from the same read) for rows that are a multiple of 128
 // elements.  A tile is `rows_per_tile` whole rows; one producer thread brings tiles in with bulk asynchronous
-// copies that complete on mbarriers (two stages), the consumer threads own 128-element segments of the tile.
-// Pass 1: segment abs-max -> shared-memory max per row; a named barrier over the consumers; pass 2: every segment
-// is scored against its row's scales (and its own group scales) from shared memory.  Chunk addresses are formed
-// by XOR, as in the multi-tensor kernel.  All waits are bounded; a consumer that gave up still meets the
-// barriers, so nobody is left waiting for it.
-constexpr int kRsStages = 2;
+// copies that complete on mbarriers (three stages, two for rows too long for that), the consumer threads own 128-element segments of the tile.
+// Pass 1: segment abs-max -> shared-memory max per row; pass 2: every segment is scored against its row's scales
+// (and its own group scales) from shared memory.  The two passes are software-pipelined: a consumer runs pass 1 of
+// tile i+1 before pass 2 of tile i, so the "all of tile i's pass 1 is done" barrier (an mbarrier the warps arrive
+// on) has normally completed long before anyone waits on it.  Chunk addresses are formed by XOR, as in the
+// multi-tensor kernel.  All waits are bounded; a consumer that gave up still arrives on every barrier, so nobody is
+// left waiting for it.
+constexpr int kRsMaxStages = 3;
 constexpr int kRsMaxRows = 8;
 constexpr int kRsMaxTileBytes = 49152;
 constexpr int kRsMaxConsumers = 256;
@@ -521,8 +523,14 @@ constexpr int kRsMaxConsumers = 256;
 struct RsParams {
     const uint16_t *x;
     long long rows, ld, n_tiles, tiles_per_cta;
-    int cols, rows_per_tile, segs_per_row, consumers, stage_bytes, grp_first;
+    int cols, rows_per_tile, segs_per_row, consumers, stage_bytes, stages, grp_first;
     RowQ rq;
+};
+
+struct RsSeg {          // what a consumer carries from pass 1 to pass 2 of a tile: up to two segments
+    uint32_t a0[2];     // shared-memory address of the segment (with the lane's XOR offset); 0 = none
+    uint32_t segmax[2];
+    int row[2];
 };
 
 template <int DT, int NI, int K0, int K1, bool GRP>
@@ -534,8 +542,8 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
     constexpr int NC = S::NC;
     constexpr int NA = NC * (GRP ? 2 : 1);
     extern __shared__ __align__(16) unsigned char smem[];   // aligned by hand below
-    __shared__ __align__(8) uint64_t full_bar[kRsStages], empty_bar[kRsStages];
-    __shared__ uint32_t rowmax[4][kRsMaxRows];
+    __shared__ __align__(8) uint64_t full_bar[kRsMaxStages], empty_bar[kRsMaxStages], row_bar[2];
+    __shared__ uint32_t rowmax[8][kRsMaxRows];
     __shared__ int err;
     __shared__ double red[33 * NA];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -543,17 +551,20 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
     const uint32_t smem_base = (smem_u32(smem) + 1023u) & ~1023u;
     unsigned char *const smem_al = smem + (smem_base - smem_u32(smem));
     if (tid == 0) {
-        for (int s = 0; s < kRsStages; ++s) {
+        for (int s = 0; s < p.stages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], n_cw);
         }
+        mbar_init(&row_bar[0], n_cw);
+        mbar_init(&row_bar[1], n_cw);
         err = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (tid < 4 * kRsMaxRows) (&rowmax[0][0])[tid] = 0;
+    if (tid < 8 * kRsMaxRows) (&rowmax[0][0])[tid] = 0;
     __syncthreads();
     const long long t_begin = (long long)blockIdx.x * p.tiles_per_cta;
     const long long t_end = min(t_begin + p.tiles_per_cta, p.n_tiles);
+    const int n_it = t_end > t_begin ? (int)(t_end - t_begin) : 0;
     const uint32_t row_bytes = (uint32_t)p.cols * 2u;
     double dacc[NA];
 #pragma unroll
@@ -563,10 +574,10 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
     if (warp == n_cw) {
         // ---------------- producer ----------------
         if (lane == 0) {
-            int it = 0;
-            for (long long t = t_begin; t < t_end; ++t, ++it) {
-                const int s = it % kRsStages;
-                const uint32_t ph = (uint32_t)(it / kRsStages) & 1u;
+            for (int it = 0; it < n_it; ++it) {
+                const long long t = t_begin + it;
+                const int s = it % p.stages;
+                const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
                 if (!mbar_wait(&empty_bar[s], ph ^ 1u, &err)) break;
                 const long long r0 = t * p.rows_per_tile;
                 const int nr = (int)min((long long)p.rows_per_tile, p.rows - r0);
@@ -580,7 +591,7 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
             }
             if (err) {
                 // give copies already issued a bounded chance to land before the shared memory is released
-                for (int s = 0; s < kRsStages; ++s) {
+                for (int s = 0; s < p.stages; ++s) {
                     const long long t0 = clock64();
                     while (!mbar_try_wait(&full_bar[s], 0) && !mbar_try_wait(&full_bar[s], 1) && clock64() - t0 < kWaitCycles) {}
                 }
@@ -589,42 +600,47 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
         }
     } else {
         // ---------------- consumers ----------------
-        int it = 0;
-        for (long long t = t_begin; t < t_end; ++t, ++it) {
-            const int s = it % kRsStages;
-            const uint32_t ph = (uint32_t)(it / kRsStages) & 1u;
+        // pass 1 of tile `it`: abs-max of this thread's segments, folded into the tile's per-row maxima
+        auto pass1 = [&](int it, RsSeg &sg) {
+            const int s = it % p.stages;
+            const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
             const bool ok = mbar_wait(&full_bar[s], ph, &err);
-            const long long r0 = t * p.rows_per_tile;
+            const long long r0 = (t_begin + it) * p.rows_per_tile;
             const int nr = (int)min((long long)p.rows_per_tile, p.rows - r0);
             const int nseg = ok ? nr * p.segs_per_row : 0;
             const uint32_t tile = smem_base + (uint32_t)s * (uint32_t)p.stage_bytes;
-            uint32_t *rmax = rowmax[it & 3];
-            uint32_t a0[2], segmax[2];
-            int srow[2];
+            uint32_t *rmax = rowmax[it & 7];
 #pragma unroll
             for (int k = 0; k < 2; ++k) {                // at most two segments per consumer (the host sizes the tile so)
-                const int sg = tid + k * p.consumers;
-                segmax[k] = 0;
-                srow[k] = 0;
-                a0[k] = 0;
-                if (sg < nseg) {
-                    srow[k] = sg / p.segs_per_row;
-                    a0[k] = tile + (uint32_t)srow[k] * row_bytes + (uint32_t)(sg - srow[k] * p.segs_per_row) * 256u + (uint32_t)((tid & 15) << 4);
+                const int g = tid + k * p.consumers;
+                sg.a0[k] = 0;
+                sg.segmax[k] = 0;
+                sg.row[k] = 0;
+                if (g < nseg) {
+                    sg.row[k] = g / p.segs_per_row;
+                    sg.a0[k] = tile + (uint32_t)sg.row[k] * row_bytes + (uint32_t)(g - sg.row[k] * p.segs_per_row) * 256u + (uint32_t)((tid & 15) << 4);
                     uint32_t m = 0;
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) m = kqmath::absmax_chunk<DT>(lds128(a0[k] ^ (uint32_t)(j << 4)), m);
-                    segmax[k] = kqmath::fold16(m);
-                    atomicMax(&rmax[srow[k]], segmax[k]);
+                    for (int j = 0; j < 16; ++j) m = kqmath::absmax_chunk<DT>(lds128(sg.a0[k] ^ (uint32_t)(j << 4)), m);
+                    sg.segmax[k] = kqmath::fold16(m);
+                    atomicMax(&rmax[sg.row[k]], sg.segmax[k]);
                 }
             }
-            asm volatile("bar.sync 1, %0;" ::"r"(p.consumers) : "memory");
-            // the buffer two tiles ahead was last read two tiles ago: everyone has left it by now
-            if (tid < kRsMaxRows) rowmax[(it + 2) & 3][tid] = 0;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&row_bar[it & 1]);
+        };
+        RsSeg cur, nxt;
+        if (n_it > 0) pass1(0, cur);
+        for (int it = 0; it < n_it; ++it) {
+            if (it + 1 < n_it) pass1(it + 1, nxt);
+            const bool ok = mbar_wait(&row_bar[it & 1], (uint32_t)(it >> 1) & 1u, &err);   // every warp has finished pass 1 of this tile
+            // the buffer four tiles ahead: nobody is within three tiles of it on either side
+            if (tid < kRsMaxRows) rowmax[(it + 4) & 7][tid] = 0;
+            const uint32_t *rmax = rowmax[it & 7];
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
-                const int sg = tid + k * p.consumers;
-                if (sg < nseg) {
-                    const uint32_t rm = rmax[srow[k]];
+                if (ok && cur.a0[k]) {
+                    const uint32_t rm = rmax[cur.row[k]];
                     if (kqmath::mag16_nonfinite<DT>(rm)) status |= MOFQ_STATUS_NONFINITE_INPUT;
                     kqmath::Sc<NC> sc;
                     S s_c, s_g;
@@ -637,14 +653,14 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
                     if (GRP) {
 #pragma unroll
                         for (int j = 0; j < NC; ++j) {
-                            if (DT == MOFQ_F16) kqmath::scale_pair_fast(kqmath::mag16_to_float<DT>(segmax[k]), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
-                            else kqmath::scale_pair(kqmath::mag16_to_float<DT>(segmax[k]), p.rq.q[j], sc.s[j], sc.inv[j], status);
+                            if (DT == MOFQ_F16) kqmath::scale_pair_fast(kqmath::mag16_to_float<DT>(cur.segmax[k]), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
+                            else kqmath::scale_pair(kqmath::mag16_to_float<DT>(cur.segmax[k]), p.rq.q[j], sc.s[j], sc.inv[j], status);
                         }
                         s_g.begin(sc);
                     }
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const uint4 v = lds128(a0[k] ^ (uint32_t)(j << 4));
+                        const uint4 v = lds128(cur.a0[k] ^ (uint32_t)(j << 4));
                         s_c.chunk(v);
                         if (GRP) s_g.chunk(v);
                     }
@@ -666,7 +682,8 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[s]);
+            if (lane == 0) mbar_arrive(&empty_bar[it % p.stages]);
+            cur = nxt;
         }
     }
     block_finish<NA>(dacc, status, hdr, partials, fin, red);
@@ -1246,24 +1263,20 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
     const mofq_tensor &x = job.x;
     const int spr = (int)(x.cols / 128);
     const int row_bytes = (int)x.cols * 2;
-    // tile shape: whole rows, at most two 128-element segments per consumer thread, consumers a multiple of 32;
-    // take the shape that keeps the most consumer lanes busy, then the one with more tiles in flight
-    int best_r = 0, best_t = 0;
-    double best_eff = 0.0;
-    for (int r = 1; r <= kRsMaxRows && (long long)r <= x.rows && r * row_bytes <= kRsMaxTileBytes; ++r) {
-        const int nseg = r * spr;
-        for (int rounds = 1; rounds <= 2; ++rounds) {
+    // tile shape: as many whole rows as fit in 36 KB (three stages of that leave room for two blocks per SM), at
+    // most two 128-element segments per consumer thread, consumers a multiple of 32
+    int best_r = 1;
+    while (best_r < kRsMaxRows && (long long)(best_r + 1) <= x.rows && (best_r + 1) * row_bytes <= 36864) ++best_r;
+    int best_t = 0;
+    for (; best_r >= 1 && !best_t; --best_r) {
+        const int nseg = best_r * spr;
+        for (int rounds = 1; rounds <= 2 && !best_t; ++rounds) {
             const int t = 32 * ((nseg + 32 * rounds - 1) / (32 * rounds));
-            if (t > kRsMaxConsumers) continue;
-            const double eff = (double)nseg / ((double)t * rounds) * (r * row_bytes <= 32768 ? 1.0 : 0.97);
-            if (eff > best_eff + 1e-9 || (eff > best_eff - 1e-9 && r * row_bytes <= 32768)) {   // ties: the larger tile up to 32 KB
-                best_eff = eff;
-                best_r = r;
-                best_t = t;
-            }
+            if (t <= kRsMaxConsumers) best_t = t;
         }
+        if (best_t) break;
     }
-    if (!best_r) return MOFQ_ERR_UNSUPPORTED;
+    if (!best_t) return MOFQ_ERR_UNSUPPORTED;
     RsParams p{};
     p.x = static_cast<const uint16_t *>(x.data);
     p.rows = x.rows;
@@ -1273,12 +1286,13 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
     p.segs_per_row = spr;
     p.consumers = best_t;
     p.stage_bytes = (best_r * row_bytes + 1023) & ~1023;
+    p.stages = 3 * p.stage_bytes + 2048 <= 113 * 1024 ? 3 : 2;   // keep two blocks per SM
     p.grp_first = (job.gran == MOFQ_PER_GROUP) ? 1 : 0;
     if (job.cs.n_int) p.rq.q[0] = job.cs.int_q;
     for (int f = 0; f < job.cs.n_fp; ++f) p.rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
     for (int j = 0; j < 3; ++j) p.rq.rq[j] = p.rq.q[j] > 0.0f ? 1.0f / p.rq.q[j] : 0.0f;
     p.n_tiles = (x.rows + best_r - 1) / best_r;
-    const size_t smem = (size_t)kRsStages * p.stage_bytes + 1024;
+    const size_t smem = (size_t)p.stages * p.stage_bytes + 1024;
     const int threads = best_t + 32;
     auto kind = [](int format) {
         return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
