@@ -5,8 +5,8 @@
 // t = RN32(x*inv), INT: RNE(t); FP: RNE of |t| onto the spacing 2^(e-M) of its binade, e clamped
 // at the smallest normal exponent (gradual underflow).  Both roundings use the add-and-subtract
 // of a power of two whose ulp equals the wanted spacing, which is an exact RNE in binary32.
-// Because every grid is symmetric, (x - v*s)^2 = (|x| - |v|*s)^2 and the scoring kernels work on
-// magnitudes only; signs matter only when codes are written out.
+// Every grid is symmetric, (x - v*s)^2 = (|x| - |v|*s)^2: the scalar kernels score magnitudes, the packed ones
+// (kq_math.cuh) keep the signs through sign-symmetric roundings; signs matter only when codes are written out.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -37,19 +37,10 @@ __device__ __forceinline__ void unpack2(uint32_t w, float &lo, float &hi)
     }
 }
 
-// 16-bit magnitude pattern -> float (exact)
-template <int DT>
-__device__ __forceinline__ float mag16_to_float(uint32_t m16)
-{
-    if (DT == MOFQ_F16) return __half2float(__ushort_as_half((unsigned short)m16));
-    return __uint_as_float(m16 << 16);
-}
-
-template <int DT>
-__device__ __forceinline__ bool mag16_nonfinite(uint32_t m16)
-{
-    return m16 >= (DT == MOFQ_F16 ? 0x7C00u : 0x7F80u);
-}
+using kqmath::fold16;
+using kqmath::mag16_nonfinite;
+using kqmath::mag16_to_float;
+using kqmath::scale_pair;
 
 // running abs-max over packed 16-bit magnitude patterns (integer order == magnitude order; Inf/NaN sort on top)
 __device__ __forceinline__ uint32_t absmax_chunk(const uint4 v, uint32_t m)
@@ -60,7 +51,6 @@ __device__ __forceinline__ uint32_t absmax_chunk(const uint4 v, uint32_t m)
     m = __vmaxu2(m, v.w & 0x7FFF7FFFu);
     return m;
 }
-__device__ __forceinline__ uint32_t fold16(uint32_t m) { return max(m & 0xFFFFu, m >> 16); }
 
 __device__ __forceinline__ void cp_async16(void *smem, const void *gmem)
 {
@@ -76,18 +66,6 @@ template <int NC>
 struct Scales {
     float s[NC], inv[NC];
 };
-
-__device__ __forceinline__ void scale_pair(float a, float Q, float &s, float &inv, int &status)
-{
-    if (a == 0.0f) {
-        s = 1.0f;
-        inv = 1.0f;
-    } else {
-        s = __fdiv_rn(a, Q);
-        inv = __fdiv_rn(Q, a);
-        if (isinf(inv)) status |= MOFQ_STATUS_SCALE_OVERFLOW;
-    }
-}
 
 template <int NI, int NFP>
 __device__ __forceinline__ void make_scales(float a, const CandSet &c, Scales<NI + NFP> &sc, int &status)
@@ -338,20 +316,20 @@ kq_score_rows(const uint16_t *__restrict__ x, long long rows, int cols, long lon
         // pass 1: abs-max per chunk
         uint32_t m16 = 0;
         for (int q = threadIdx.x; q < chunks; q += kRowThreads) {
-            const uint32_t c16 = kqmath::fold16(kqmath::absmax_chunk<DT>(row4[q], 0u));
+            const uint32_t c16 = fold16(kqmath::absmax_chunk<DT>(row4[q], 0u));
             if (GRP) cmax[q] = (uint16_t)c16;
             m16 = max(m16, c16);
         }
-        if (kqmath::mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+        if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
         if (GRP) {
             __syncthreads();
             for (int g = threadIdx.x; g < gpr; g += kRowThreads) {
                 uint32_t gm = 0;
                 for (int j = 0; j < (1 << cpg_shift); ++j) gm = max(gm, (uint32_t)cmax[(g << cpg_shift) + j]);
-                const float a = kqmath::mag16_to_float<DT>(gm);
+                const float a = mag16_to_float<DT>(gm);
                 kqmath::Sc<NC> sc;
 #pragma unroll
-                for (int j = 0; j < NC; ++j) kqmath::scale_pair(a, rq.q[j], sc.s[j], sc.inv[j], status);
+                for (int j = 0; j < NC; ++j) scale_pair(a, rq.q[j], sc.s[j], sc.inv[j], status);
                 gsc[g] = sc;
             }
         }
@@ -361,7 +339,7 @@ kq_score_rows(const uint16_t *__restrict__ x, long long rows, int cols, long lon
                 int st = 0;
                 kqmath::Sc<NC> sc;
 #pragma unroll
-                for (int j = 0; j < NC; ++j) kqmath::scale_pair(kqmath::mag16_to_float<DT>(rm), rq.q[j], sc.s[j], sc.inv[j], st);
+                for (int j = 0; j < NC; ++j) scale_pair(mag16_to_float<DT>(rm), rq.q[j], sc.s[j], sc.inv[j], st);
                 row_sc = sc;
                 row_status = st;
             }
@@ -459,13 +437,13 @@ kq_select_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long 
         } else if (live) {
             for (int q = tl; q < cpb; q += team) m = kqmath::absmax_chunk<DT>(__ldg(blk + q), m);
         }
-        uint32_t m16 = kqmath::fold16(m);
+        uint32_t m16 = fold16(m);
         for (int o = team >> 1; o; o >>= 1) m16 = max(m16, __shfl_xor_sync(0xffffffffu, m16, o));
-        if (kqmath::mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
-        const float a = kqmath::mag16_to_float<DT>(m16);
+        if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+        const float a = mag16_to_float<DT>(m16);
         kqmath::Sc<NC> sc;
 #pragma unroll
-        for (int j = 0; j < NC; ++j) kqmath::scale_pair(a, rq.q[j], sc.s[j], sc.inv[j], status);
+        for (int j = 0; j < NC; ++j) scale_pair(a, rq.q[j], sc.s[j], sc.inv[j], status);
         S scorer;
         scorer.begin(sc);
         if (one_pass) {
@@ -622,7 +600,7 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
                     uint32_t m = 0;
 #pragma unroll
                     for (int j = 0; j < 16; ++j) m = kqmath::absmax_chunk<DT>(lds128(sg.a0[k] ^ (uint32_t)(j << 4)), m);
-                    sg.segmax[k] = kqmath::fold16(m);
+                    sg.segmax[k] = fold16(m);
                     atomicMax(&rmax[sg.row[k]], sg.segmax[k]);
                 }
             }
@@ -641,20 +619,20 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
             for (int k = 0; k < 2; ++k) {
                 if (ok && cur.a0[k]) {
                     const uint32_t rm = rmax[cur.row[k]];
-                    if (kqmath::mag16_nonfinite<DT>(rm)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+                    if (mag16_nonfinite<DT>(rm)) status |= MOFQ_STATUS_NONFINITE_INPUT;
                     kqmath::Sc<NC> sc;
                     S s_c, s_g;
 #pragma unroll
                     for (int j = 0; j < NC; ++j) {
-                        if (DT == MOFQ_F16) kqmath::scale_pair_fast(kqmath::mag16_to_float<DT>(rm), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
-                        else kqmath::scale_pair(kqmath::mag16_to_float<DT>(rm), p.rq.q[j], sc.s[j], sc.inv[j], status);
+                        if (DT == MOFQ_F16) kqmath::scale_pair_fast(mag16_to_float<DT>(rm), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
+                        else scale_pair(mag16_to_float<DT>(rm), p.rq.q[j], sc.s[j], sc.inv[j], status);
                     }
                     s_c.begin(sc);
                     if (GRP) {
 #pragma unroll
                         for (int j = 0; j < NC; ++j) {
-                            if (DT == MOFQ_F16) kqmath::scale_pair_fast(kqmath::mag16_to_float<DT>(cur.segmax[k]), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
-                            else kqmath::scale_pair(kqmath::mag16_to_float<DT>(cur.segmax[k]), p.rq.q[j], sc.s[j], sc.inv[j], status);
+                            if (DT == MOFQ_F16) kqmath::scale_pair_fast(mag16_to_float<DT>(cur.segmax[k]), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
+                            else scale_pair(mag16_to_float<DT>(cur.segmax[k]), p.rq.q[j], sc.s[j], sc.inv[j], status);
                         }
                         s_g.begin(sc);
                     }
