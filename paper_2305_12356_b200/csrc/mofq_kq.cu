@@ -978,35 +978,163 @@ __device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
     return d & 0xFFu;
 }
 
+// ---- fast code emission for group and per-tensor scales (codes + scales only, abs-max scales) -------------------
+// A team of lanes owns one scale block (a group; for a per-tensor scale a run of 32 elements), each lane four
+// consecutive 16-byte chunks held in registers: abs-max by shuffles inside the team, the scale pair, then the codes
+// through packed f32x2 arithmetic and the hardware converts, stored as contiguous runs per lane.  The format is
+// decoded once per kernel (it may have been picked on the device), not per element.
+enum { CLS_INT4 = 0, CLS_INT8 = 1, CLS_E2M1 = 2, CLS_E4M3 = 3, CLS_E5M2 = 4 };
+
+template <int DT, int CLS>
+__device__ __forceinline__ uint2 chunk_codes(const uint4 v, uint64_t inv2)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t c[4];  // CLS with 8-bit codes: 16 bits per word; 4-bit codes: 8 bits per word
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint64_t a2 = kqmath::unpack2<DT>(w[i]);
+        float lo, hi;
+        if (CLS == CLS_INT4 || CLS == CLS_INT8) {
+            // t = RN32(x * inv) first (the code is decided on the rounded t), then the low mantissa bits of
+            // t + 1.5 * 2^23 are the two's-complement code
+            // (the add stays scalar: a packed multiply followed by a packed add came out as one fused operation,
+            // which rounds the exact product instead of t and breaks ties differently)
+            kqmath::upk(kqmath::mul2(a2, inv2), lo, hi);
+            lo = __fadd_rn(lo, kMagic);
+            hi = __fadd_rn(hi, kMagic);
+            uint32_t t = __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x0040);
+            if (CLS == CLS_INT4) {
+                t &= 0x0F0Fu;
+                t = (t | (t >> 4)) & 0xFFu;
+            }
+            c[i] = t;
+        } else {
+            kqmath::upk(kqmath::mul2(a2, inv2), lo, hi);
+            c[i] = CLS == CLS_E2M1 ? cvt_e2m1x2(lo, hi) : CLS == CLS_E4M3 ? cvt_e4m3x2(lo, hi) : cvt_e5m2x2(lo, hi);
+        }
+    }
+    uint2 o;
+    if (CLS == CLS_INT4 || CLS == CLS_E2M1) {
+        o.x = __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
+        o.y = 0;
+    } else {
+        o.x = __byte_perm(c[0], c[1], 0x5410);
+        o.y = __byte_perm(c[2], c[3], 0x5410);
+    }
+    return o;
+}
+
+template <int DT, int CLS>
+__device__ __forceinline__ void emit_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, float Q, int width,
+                                            bool uniform, unsigned char *codes_out, float *scales_out, WsHeader *hdr, int &status)
+{
+    constexpr int KPL = 4;
+    constexpr bool kFour = CLS == CLS_INT4 || CLS == CLS_E2M1;
+    const int lane = threadIdx.x & 31;
+    const int cpb = width >> 3;                             // chunks per block: 1, 2, 4, ..., 32
+    const int n_k = min(KPL, cpb);                          // chunks per lane
+    const int team = max(1, cpb / KPL);
+    const int tl = lane & (team - 1);
+    const int teams_per_warp = 32 / team;
+    const int per_row = cols / width;
+    const long long n_blocks = rows * per_row;
+    const long long warp_id = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const long long n_warps = (long long)gridDim.x * (blockDim.x >> 5);
+    const float rQ = 1.0f / Q;
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(codes_out) & 15) == 0;   // blocks of >= 32 elements start on 32-element boundaries
+    float s_u = 1.0f, inv_u = 1.0f;
+    if (uniform) {
+        const uint32_t m16 = *reinterpret_cast<volatile uint32_t *>(&hdr->absmax_bits);
+        if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+        scale_pair(mag16_to_float<DT>(m16), Q, s_u, inv_u, status);
+        if (scales_out && blockIdx.x == 0 && threadIdx.x == 0) scales_out[0] = s_u;
+    }
+    for (long long b0 = warp_id * teams_per_warp; b0 < n_blocks; b0 += n_warps * teams_per_warp) {
+        const long long b = b0 + lane / team;
+        const bool live = b < n_blocks;                     // whole teams are live or not; shuffles stay warp-wide
+        const long long r = live ? b / per_row : 0;
+        const long long c0 = live ? (b - r * per_row) * width : 0;
+        const uint4 *blk = reinterpret_cast<const uint4 *>(x + r * ld + c0);
+        uint4 v[KPL];
+        uint32_t m = 0;
+#pragma unroll
+        for (int k = 0; k < KPL; ++k) {
+            v[k] = (live && k < n_k) ? __ldg(blk + tl * n_k + k) : make_uint4(0, 0, 0, 0);
+            m = kqmath::absmax_chunk<DT>(v[k], m);
+        }
+        float s = s_u, inv = inv_u;
+        if (!uniform) {
+            uint32_t m16 = fold16(m);
+            for (int o = team >> 1; o; o >>= 1) m16 = max(m16, __shfl_xor_sync(0xffffffffu, m16, o));
+            if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+            const float a = mag16_to_float<DT>(m16);
+            if (DT == MOFQ_F16) kqmath::scale_pair_fast(a, Q, rQ, s, inv);
+            else scale_pair(a, Q, s, inv, status);
+            if (live && tl == 0 && scales_out) scales_out[b] = s;
+        }
+        if (!live) continue;
+        const uint64_t inv2 = kqmath::pk(inv, inv);
+        const size_t e0 = (size_t)r * cols + (size_t)c0 + (size_t)(tl * n_k) * 8;   // first element of this lane's run
+        if (n_k == KPL && vec_ok) {
+            // a lane's four chunks are one aligned run of 16 (4-bit) or 32 (8-bit) bytes of codes
+            uint2 o[KPL];
+#pragma unroll
+            for (int k = 0; k < KPL; ++k) o[k] = chunk_codes<DT, CLS>(v[k], inv2);
+            if (kFour) {
+                *reinterpret_cast<uint4 *>(codes_out + (e0 >> 1)) = make_uint4(o[0].x, o[1].x, o[2].x, o[3].x);
+            } else {
+                reinterpret_cast<uint4 *>(codes_out + e0)[0] = make_uint4(o[0].x, o[0].y, o[1].x, o[1].y);
+                reinterpret_cast<uint4 *>(codes_out + e0)[1] = make_uint4(o[2].x, o[2].y, o[3].x, o[3].y);
+            }
+            continue;
+        }
+#pragma unroll
+        for (int k = 0; k < KPL; ++k) {
+            if (k < n_k) {
+                const uint2 o = chunk_codes<DT, CLS>(v[k], inv2);
+                if (kFour) reinterpret_cast<uint32_t *>(codes_out + (e0 >> 1))[k] = o.x;
+                else reinterpret_cast<uint2 *>(codes_out + e0)[k] = o;
+            }
+        }
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256)
+kq_emit_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, FmtDesc f, int width, int uniform,
+               unsigned char *codes_out, float *scales_out, WsHeader *hdr, const EmitSel sel)
+{
+    if (sel.res) {  // the winner of the selection record decides the grid
+        const int c = min(max(sel.res->chosen, 0), MOFQ_MAX_CAND - 1);
+        f = sel.cand[c];
+        if (sel.tag_out && blockIdx.x == 0 && threadIdx.x == 0) *sel.tag_out = sel.format[c];
+    }
+    int status = 0;
+    const int cls = !f.is_fp ? (f.bits == 4 ? CLS_INT4 : CLS_INT8) : f.M == 1 ? CLS_E2M1 : f.M == 3 ? CLS_E4M3 : CLS_E5M2;
+    switch (cls) {
+    case CLS_INT4: emit_blocks<DT, CLS_INT4>(x, rows, cols, ld, f.Q, width, uniform != 0, codes_out, scales_out, hdr, status); break;
+    case CLS_INT8: emit_blocks<DT, CLS_INT8>(x, rows, cols, ld, f.Q, width, uniform != 0, codes_out, scales_out, hdr, status); break;
+    case CLS_E2M1: emit_blocks<DT, CLS_E2M1>(x, rows, cols, ld, f.Q, width, uniform != 0, codes_out, scales_out, hdr, status); break;
+    case CLS_E4M3: emit_blocks<DT, CLS_E4M3>(x, rows, cols, ld, f.Q, width, uniform != 0, codes_out, scales_out, hdr, status); break;
+    default: emit_blocks<DT, CLS_E5M2>(x, rows, cols, ld, f.Q, width, uniform != 0, codes_out, scales_out, hdr, status); break;
+    }
+    if (status) atomicOr(&hdr->status, status);
+}
+
 // codes of 8 consecutive elements for one format, packed little-endian (8-bit: 64 bits, 4-bit: 32 bits)
 template <int DT>
 __device__ __forceinline__ uint64_t codes8(const uint4 v, int format, float inv)
 {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint64_t out = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float lo, hi;
-        unpack2<DT>(w[i], lo, hi);
-        const float tl = __fmul_rn(lo, inv), th = __fmul_rn(hi, inv);
-        uint32_t c;  // two codes
-        int bits;
-        switch (format) {
-        case MOFQ_FP8_E4M3: c = cvt_e4m3x2(tl, th); bits = 8; break;
-        case MOFQ_FP8_E5M2: c = cvt_e5m2x2(tl, th); bits = 8; break;
-        case MOFQ_INT8:
-            c = (__float_as_uint(__fadd_rn(tl, kMagic)) & 0xFFu) | ((__float_as_uint(__fadd_rn(th, kMagic)) & 0xFFu) << 8);
-            bits = 8;
-            break;
-        case MOFQ_INT4:
-            c = (__float_as_uint(__fadd_rn(tl, kMagic)) & 0xFu) | ((__float_as_uint(__fadd_rn(th, kMagic)) & 0xFu) << 4);
-            bits = 4;
-            break;
-        default: c = cvt_e2m1x2(tl, th); bits = 4; break;  // both E2M1 variants: same spacing below the IEEE maximum 3
-        }
-        out |= (uint64_t)c << (i * 2 * bits);
+    const uint64_t inv2 = kqmath::pk(inv, inv);
+    uint2 o;
+    switch (format) {  // uniform over the launch; the per-class code below is branch-free
+    case MOFQ_INT4: o = chunk_codes<DT, CLS_INT4>(v, inv2); break;
+    case MOFQ_INT8: o = chunk_codes<DT, CLS_INT8>(v, inv2); break;
+    case MOFQ_FP8_E4M3: o = chunk_codes<DT, CLS_E4M3>(v, inv2); break;
+    case MOFQ_FP8_E5M2: o = chunk_codes<DT, CLS_E5M2>(v, inv2); break;
+    default: o = chunk_codes<DT, CLS_E2M1>(v, inv2); break;  // both E2M1 variants: same spacing below the IEEE maximum 3
     }
-    return out;
+    return (uint64_t)o.x | ((uint64_t)o.y << 32);
 }
 
 struct EmitSet {
@@ -1473,6 +1601,23 @@ int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, con
         else
             kq_absmax<1><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, hdr);
         MOFQ_CUDA_OK(cudaGetLastError());
+    }
+    if ((gran == MOFQ_PER_GROUP || gran == MOFQ_PER_TENSOR) && !scales_in && codes_out && !dequant_out && !values_out &&
+        (gran == MOFQ_PER_GROUP || x.cols % 32 == 0)) {
+        // codes + scales under abs-max scales: the register-resident team kernel
+        const int width = gran == MOFQ_PER_GROUP ? group : 32;
+        const int team = std::max(1, (width >> 3) / 4);
+        const long long n_blocks = x.rows * (x.cols / width);
+        const long long warps = (n_blocks + (32 / team) - 1) / (32 / team);
+        const int g = (int)std::min<long long>((warps + 7) / 8, (long long)nsm * 8);
+        if (x.dtype == MOFQ_F16)
+            kq_emit_blocks<0><<<g, 256, 0, st>>>(xp, x.rows, (int)x.cols, x.ld, f, width, gran == MOFQ_PER_TENSOR,
+                                                 (unsigned char *)codes_out, scales_out, hdr, es);
+        else
+            kq_emit_blocks<1><<<g, 256, 0, st>>>(xp, x.rows, (int)x.cols, x.ld, f, width, gran == MOFQ_PER_TENSOR,
+                                                 (unsigned char *)codes_out, scales_out, hdr, es);
+        MOFQ_CUDA_OK(cudaGetLastError());
+        return MOFQ_OK;
     }
     const int grid = (int)std::min<long long>(x.rows, (long long)nsm * 8);
 #define MOFQ_EMIT(DT_, G_)                                                                                                   \

@@ -387,3 +387,38 @@ def test_fast_scale_pair_is_correctly_rounded_for_every_binary16_magnitude(orc, 
     for k in (0, 1, 2, 1000, 0x3C00, 0x7BFF):                                    # and the oracle's own routine on a few
         so, io = orc.scale_from_absmax(getattr(orc, name), a[k])
         assert so == want_s[k] and io == want_i[k]
+
+
+# ---- codes + scales only: the register-resident emission kernel (group and per-tensor scales) ---------------------------------
+def _check_codes_only(orc, x, name, gran, group=0):
+    fmt_o = getattr(orc, name)
+    bits = orc.format_bits(fmt_o)
+    got = mofq.quantize_tensor(x, name, gran, group)
+    want = orc.quantize(host(x).contiguous(), fmt_o, orc_gran(orc, gran), group)
+    np.testing.assert_array_equal(unpack_codes(got["codes"], bits, x.numel()), want["codes"].reshape(-1))
+    np.testing.assert_array_equal(got["scales"].cpu().numpy().view(np.uint32), want["scales"].view(np.uint32))
+    assert int(got["status"].item()) == 0
+
+
+@pytest.mark.parametrize("name", FMT4 + FMT8)
+@pytest.mark.parametrize("gran,group", [("group", 128), ("group", 256), ("group", 32), ("group", 16), ("group", 8), ("tensor", 0)])
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_codes_only_emission_matches_oracle(orc, dev, name, gran, group, dtype):
+    x = _weights(dev, 301, 1280, seed=51, layer=2, dtype=dtype)                  # 301 rows: ragged against the warp teams
+    x[5, 100:228] = 0                                                             # an all-zero group
+    x[9, 3] = -0.0
+    _check_codes_only(orc, x, name, gran, group)
+
+
+def test_codes_only_emission_strided_and_every_fp16_pattern(orc, dev):
+    full = _weights(dev, 40, 1024 + 64, seed=52)
+    view = full[:, 32:1056]
+    for name in ("INT4", "FP4_E2M1", "INT8", "FP8_E5M2"):
+        _check_codes_only(orc, view, name, "group", 128)
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    bits = bits[(bits & 0x7C00) != 0x7C00]
+    bits = np.concatenate([bits, np.zeros((-bits.size) % 1024, np.uint16)])
+    x = torch.from_numpy(bits.view(np.int16).copy()).view(torch.float16).reshape(-1, 1024).to(dev)
+    for name in FMT4 + FMT8:
+        for gran, group in (("group", 128), ("group", 8), ("tensor", 0)):
+            _check_codes_only(orc, x, name, gran, group)
