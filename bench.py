@@ -307,6 +307,22 @@ def main():
             samples.append(b0.elapsed_time(b1))
         burst_ms = sorted(samples)[len(samples) // 2]
 
+    # Algorithm 1's last step, for context (not part of the metric): every layer quantised to its winner, read on
+    # the device from the records the last step left
+    emit_ms = None
+    if rank == 0 and not layer_metric and not streaming and len(grans) == 1 and fp16_bytes < 40e9:
+        bufs = B.EmitBuffers(prepared, cfg)
+        mofq.emit_selected(prepared, cfg, results, buffers=bufs)
+        torch.cuda.synchronize()
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        q0.record()
+        mofq.emit_selected(prepared, cfg, results, buffers=bufs)
+        q1.record()
+        torch.cuda.synchronize()
+        emit_ms = q0.elapsed_time(q1)
+        assert int(bufs.ws[:4].view(torch.int32).item()) == 0
+        del bufs
+
     # decisions (for the record) and a sanity check that the step produced them
     recs = B._parse_results(bytes(results.cpu().numpy()), n_rec, cfg.n_candidates)
     assert all(r["status"] == 0 and 0 <= r["chosen"] < cfg.n_candidates for r in recs)
@@ -367,7 +383,7 @@ def main():
                        "candidates": list(wl["candidates"]), "granularity": list(grans), "group": wl["group"],
                        "criterion": wl["metric"], "tokens": T, "streaming_synthesis": streaming, "synthesis_ms_per_step": synth_ms,
                        "l2": "inputs larger than L2" if fp16_bytes > 2.5e8 else "inputs fit in L2",
-                       "model_select_time_ms": ms_per_step, "fp_share": fp_share, "min_rel_margin": min_margin},
+                       "model_select_time_ms": ms_per_step, "emit_winners_ms": emit_ms, "fp_share": fp_share, "min_rel_margin": min_margin},
             "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * launches_per_step, "roofline": roofline,
         }
         if layer_metric:

@@ -353,31 +353,40 @@ class MofqPacked(C.Structure):
     _fields_ = [("codes", C.c_void_p), ("scales", C.c_void_p)]
 
 
-def emit_selected(layers, cfg, results):
+class EmitBuffers:
+    """Preallocated destinations of emit_selected for a layer list (codes, scales, format tags, status word)."""
+
+    def __init__(self, layers, cfg):
+        prep = prepare_layers(layers)
+        dev = prep.device
+        n = len(prep)
+        self.array = (MofqPacked * n)()
+        self.packed = []
+        for i, layer in enumerate(prep.layers):
+            W = layer if torch.is_tensor(layer) else layer[0]
+            rows, cols = W.shape
+            codes = torch.empty(rows * cols * cfg.bit_width // 8, dtype=torch.uint8, device=dev)
+            scales = torch.empty(n_scales(cfg.w_gran, rows, cols, cfg.w_group), dtype=torch.float32, device=dev)
+            self.array[i].codes, self.array[i].scales = codes.data_ptr(), scales.data_ptr()
+            self.packed.append(dict(codes=codes, scales=scales))
+        self.formats = torch.empty(n, dtype=torch.int32, device=dev)
+        self.ws = _workspace(256, dev)
+
+
+def emit_selected(layers, cfg, results, buffers=None):
     """mofq_emit_selected: quantise every layer's W to the format its selection record names (read on the device).
 
     `results` is the raw device byte tensor of select_formats(..., parse=False).  Returns (packed, formats, status):
     packed = list of dict(codes uint8 tensor, scales float32 tensor) per layer, formats = int32 device tensor of
-    mofq_format tags, status = 1-element int32 device tensor.  Nothing synchronises.
+    mofq_format tags, status = 1-element int32 device tensor.  Nothing synchronises.  Pass an EmitBuffers to reuse
+    the destinations across calls.
     """
     L = lib()
     prep = prepare_layers(layers)
-    dev = prep.device
-    n = len(prep)
-    out = (MofqPacked * n)()
-    packed = []
-    for i, layer in enumerate(prep.layers):
-        W = layer if torch.is_tensor(layer) else layer[0]
-        rows, cols = W.shape
-        codes = torch.empty(rows * cols * cfg.bit_width // 8, dtype=torch.uint8, device=dev)
-        scales = torch.empty(n_scales(cfg.w_gran, rows, cols, cfg.w_group), dtype=torch.float32, device=dev)
-        out[i].codes, out[i].scales = codes.data_ptr(), scales.data_ptr()
-        packed.append(dict(codes=codes, scales=scales))
-    formats = torch.empty(n, dtype=torch.int32, device=dev)
-    ws = _workspace(256, dev)
-    _check(L.mofq_emit_selected(prep.array, n, C.byref(cfg), results.data_ptr(), C.cast(out, C.c_void_p), formats.data_ptr(),
-                                ws.data_ptr(), ws.numel(), _stream(dev)))
-    return packed, formats, ws[:4].view(torch.int32)
+    b = buffers if buffers is not None else EmitBuffers(prep, cfg)
+    _check(L.mofq_emit_selected(prep.array, len(prep), C.byref(cfg), results.data_ptr(), C.cast(b.array, C.c_void_p),
+                                b.formats.data_ptr(), b.ws.data_ptr(), b.ws.numel(), _stream(prep.device)))
+    return b.packed, b.formats, b.ws[:4].view(torch.int32)
 
 
 def select_formats_host(layers, cfg, device, workspace=None):
