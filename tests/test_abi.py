@@ -105,3 +105,38 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "libmofq.so"))
     with pytest.raises(B.MofqError):
         B.lib()
+
+
+def test_added_entry_points_validate_their_arguments():
+    L = mofq.lib()
+    d = _desc()
+    fm = (C.c_int32 * 2)(B.INT4, B.FP4_E2M1)
+    vp = C.c_void_p
+    # block-wise selection: channel or group only, at most three candidates, outputs required
+    assert L.mofq_select_blocks(C.byref(d), fm, 2, B.PER_TENSOR, 0, vp(0x50000), None, vp(0x30000), vp(0x20000), 1 << 20, None) == -2
+    assert L.mofq_select_blocks(C.byref(d), fm, 2, B.PER_CHANNEL, 0, None, None, vp(0x30000), vp(0x20000), 1 << 20, None) == -1
+    assert L.mofq_select_blocks(C.byref(d), fm, 2, B.PER_GROUP, 96, vp(0x50000), None, vp(0x30000), vp(0x20000), 1 << 20, None) == -2
+    four = (C.c_int32 * 4)(B.INT4, B.FP4_E2M1, B.FP4_E2M1_IEEE, B.INT4)
+    assert L.mofq_select_blocks(C.byref(d), four, 4, B.PER_CHANNEL, 0, vp(0x50000), None, vp(0x30000), vp(0x20000), 1 << 20, None) == -1
+    assert L.mofq_select_blocks(C.byref(d), fm, 2, B.PER_CHANNEL, 0, vp(0x50000), None, vp(0x30000), vp(0x20000), 64, None) == -4
+    # calibration scales
+    assert L.mofq_absmax_update(C.byref(d), None, None) == -1
+    assert L.mofq_absmax_update(C.byref(_desc(ptr=0)), vp(0x30000), None) == -1
+    assert L.mofq_tensor_error_scaled(C.byref(d), fm, 2, None, vp(0x30000), vp(0x20000), 1 << 20, None) == -1
+    assert L.mofq_tensor_error_scaled(C.byref(d), fm, 0, vp(0x60000), vp(0x30000), vp(0x20000), 1 << 20, None) == -1
+    mixed = (C.c_int32 * 2)(B.INT4, B.FP8_E4M3)
+    assert L.mofq_tensor_error_scaled(C.byref(d), mixed, 2, vp(0x60000), vp(0x30000), vp(0x20000), 1 << 20, None) == -2
+    # emission of the selected formats
+    cfg = mofq.make_config(4, ["INT4", "FP4_E2M1"], w_gran="group", w_group=128)
+    layers = (B.MofqLayer * 1)()
+    layers[0].W = _desc()
+    out = (B.MofqPacked * 1)()
+    assert L.mofq_emit_selected(layers, 1, C.byref(cfg), vp(0x40000), out, None, vp(0x20000), 256, None) == -1   # NULL destinations
+    out[0].codes, out[0].scales = 0x70000, 0x80000
+    assert L.mofq_emit_selected(layers, 1, C.byref(cfg), None, out, None, vp(0x20000), 256, None) == -1
+    assert L.mofq_emit_selected(layers, 1, C.byref(cfg), vp(0x40000), out, None, vp(0x20000), 16, None) == -4
+    bad = mofq.make_config(4, ["INT4", "FP4_E2M1"], w_gran="group", w_group=96)
+    assert L.mofq_emit_selected(layers, 1, C.byref(bad), vp(0x40000), out, None, vp(0x20000), 256, None) == -2
+    # diagnostics
+    assert L.mofq_diag_scale_pair(B.INT4, None, vp(0x30000), vp(0x30100), 4, None) == -1
+    assert L.mofq_diag_scale_pair(77, vp(0x20000), vp(0x30000), vp(0x30100), 4, None) == -1
