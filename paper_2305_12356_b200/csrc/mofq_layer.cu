@@ -32,7 +32,8 @@ constexpr int BM = 128;
 constexpr int kRowBytes = 128;  // bytes of K per tile row: 64 16-bit or 128 8-bit elements (one 128-byte swizzle row)
 constexpr int kABytes = BM * kRowBytes;
 constexpr int kRingBytes = 192 * 1024;
-constexpr int kGemmThreads = 192;  // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-5: epilogue
+constexpr int kEpiWarps = 8;        // two per tensor-memory lane quarter, each on half of the tile's columns
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;  // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2..: epilogue
 // Tile width BN is 128 or 256: the wider tile moves 25% fewer operand bytes per flop (the main loop is bound by
 // L2 -> shared-memory traffic), the narrower one quantises better onto 148 SMs.  Two accumulators of BN columns.
 // CG = 2: a cluster of two CTAs computes a 256 x BN tile; each CTA stages its own 128 rows of A and BN/2 rows of B
@@ -148,6 +149,7 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, ui
 }
 
 // 32 lanes x 32 consecutive fp32 columns: thread i receives row (lane base + i)
+// issues the load; the data is valid after tc_ld_wait
 __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -158,7 +160,18 @@ __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
                    "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
                    "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// completes every tensor-memory load this thread has issued; the registers are operands so that no use of them can
+// be scheduled ahead of the wait
+__device__ __forceinline__ void tc_ld_wait(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                   "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                   "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                   "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :
+                 : "memory");
 }
 
 // Shared-memory matrix descriptor for a K-major tile whose rows are 128 bytes (64 16-bit elements) written
@@ -194,7 +207,7 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], tfull_bar[2], tempty_bar[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int err_flag;
-    __shared__ double red[4];
+    __shared__ double red[kEpiWarps];
     volatile int *const perr = &err_flag;
 #define err (*perr)
 
@@ -214,10 +227,10 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&tfull_bar[b], 1);
-            mbar_init(&tempty_bar[b], 4 * CG);  // the epilogue warps of every CTA of the unit release the leader
+            mbar_init(&tempty_bar[b], kEpiWarps * CG);  // the epilogue warps of every CTA of the unit release the leader
         }
         err = 0;
-        red[0] = red[1] = red[2] = red[3] = 0.0;
+        for (int i = 0; i < kEpiWarps; ++i) red[i] = 0.0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // the MMA warp owns the tensor-memory allocation
@@ -328,18 +341,21 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
     } else {
         // ---------------- epilogue: warps 2..5 read the lane quarter (warp % 4) of the accumulator ----------------
+        // The epilogue is bound by the latency of its tensor-memory and global loads, not by arithmetic: eight warps
+        // keep twice as many of them in flight as four would.
         const int q = warp & 3;
+        const int half = (warp - 2) >> 2;                 // which half of the tile's columns this warp handles
+        constexpr int kChunks = BN / 32 / (kEpiWarps / 4);
         const float alpha = *p.alpha;
         double dsum = 0.0;
         int local = 0;
         for (int tile = unit; tile < n_tiles; tile += n_units, ++local) {
             const int buf = local & 1;
             const int m0 = (tile % tiles_m) * BM * CG + rank * BM, n0 = (tile / tiles_m) * BN;
-            if (!mbar_wait(&tfull_bar[buf], (local >> 1) & 1, perr)) break;
-            tc_fence_after();
             const int row = m0 + q * 32 + lane;
             float fsum = 0.0f;
-            // the stored Y of the next 32-column chunk is fetched while the current chunk is processed
+            // the stored Y of the next 32-column chunk is fetched while the current chunk is processed; the first
+            // chunk's is requested before the accumulator is waited for
             const bool vec = (p.N & 3) == 0;
             float4 ycur[8], ynext[8];
             auto prefetch_y = [&](int c, float4 (&y)[8]) {
@@ -350,12 +366,21 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     for (int j = 0; j < 8; ++j) y[j] = __ldg(src + j);
                 }
             };
-            prefetch_y(0, ycur);
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                if (c + 1 < BN / 32) prefetch_y(c + 1, ynext);
-                uint32_t r[32];
-                tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), r);
+            prefetch_y(half * kChunks, ycur);
+            if (!mbar_wait(&tfull_bar[buf], (local >> 1) & 1, perr)) break;
+            tc_fence_after();
+            // two register sets: the tensor-memory load of chunk c+1 is in flight while chunk c is processed
+            uint32_t ra[32], rb[32];
+            const uint32_t t0 = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
+            tc_ld_32x32(t0 + (uint32_t)(half * kChunks * 32), ra);
+#pragma unroll
+            for (int ci = 0; ci < kChunks; ++ci) {
+                const int c = half * kChunks + ci;
+                uint32_t(&r)[32] = (ci & 1) ? rb : ra;
+                uint32_t(&rn)[32] = (ci & 1) ? ra : rb;
+                if (ci + 1 < kChunks) prefetch_y(c + 1, ynext);
+                tc_ld_wait(r);
+                if (ci + 1 < kChunks) tc_ld_32x32(t0 + (uint32_t)((c + 1) * 32), rn);
                 const int col0 = n0 + c * 32;
                 if (p.kind == KIND_I8) {  // exact integer dot products -> float
 #pragma unroll
@@ -392,7 +417,9 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             }
                         }
                     } else {
-                        for (int j = 0; j < 32 && col0 + j < p.N; ++j) {  // ragged right edge
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {  // ragged right edge (static indices keep r in registers)
+                            if (col0 + j >= p.N) continue;
                             const float a = __uint_as_float(r[j]);
                             if (p.mode == 0) {
                                 const float v = a * alpha;
@@ -419,13 +446,15 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
-        if (lane == 0) red[q] = dsum;
+        if (lane == 0) red[warp - 2] = dsum;
     }
     tc_fence_before();
     if (CG == 2) cluster_sync();  // no CTA leaves while its peer may still touch its shared or tensor memory
     else __syncthreads();
     if (threadIdx.x == 0) {
-        p.partials[blockIdx.x] = (red[0] + red[1]) + (red[2] + red[3]);
+        double tot = 0.0;
+        for (int i = 0; i < kEpiWarps; ++i) tot += red[i];
+        p.partials[blockIdx.x] = tot;
         if (err) atomicOr(p.status, MOFQ_STATUS_TIMEOUT);
     }
     if (warp == 1) {
