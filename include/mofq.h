@@ -53,7 +53,7 @@ typedef enum {
 } mofq_format;
 
 /* Scale granularity (Section 3.2: per-channel weights, per-tensor activations; per-group =
- * `group` consecutive elements along the input dimension, cols % group == 0, group % 8 == 0). */
+ * `group` consecutive elements along the input dimension: a power of two in [8, 256] that divides cols). */
 typedef enum { MOFQ_PER_TENSOR = 0, MOFQ_PER_CHANNEL = 1, MOFQ_PER_GROUP = 2 } mofq_gran;
 #define MOFQ_GRAN_NONE (-1)
 
