@@ -271,6 +271,14 @@ size_t mofq_noalloc_scratch_bytes(void);
 int mofq_diag_fp_round(int format, const float *t, float *out, int64_t n, void *stream);
 
 /*
+ * mofq_diag_wait_expiry - diagnostic: runs the bounded wait that every pipelined kernel of the library uses on a
+ * barrier that nothing will ever complete.  The wait gives up after about two seconds, the kernel returns and
+ * *status_out (device int32) holds MOFQ_STATUS_TIMEOUT: a broken pipeline ends as a status bit, not as a hung GPU.
+ * (The paper has no counterpart; this exists so that a test can show it.)
+ */
+int mofq_diag_wait_expiry(int32_t *status_out, void *stream);
+
+/*
  * mofq_diag_scale_pair - diagnostic: scale = RN32(a / Q) and inv = RN32(Q / a) (Section 3.2: abs-max scaling; a = 0
  * gives 1, 1) as the multi-tensor scoring kernel computes them for binary16 tensors, i.e. without the general
  * division routine.  Valid for abs-max values a binary16 tensor can have (0 or 2^-24 ... 65504); a test compares

@@ -81,6 +81,8 @@ def lib():
         L.mofq_absmax_update.argtypes = [C.POINTER(MofqTensor), vp, vp]
         L.mofq_tensor_error_scaled.restype = C.c_int
         L.mofq_tensor_error_scaled.argtypes = [C.POINTER(MofqTensor), C.POINTER(C.c_int32), C.c_int, vp, vp, vp, sz, vp]
+        L.mofq_diag_wait_expiry.restype = C.c_int
+        L.mofq_diag_wait_expiry.argtypes = [vp, vp]
         L.mofq_diag_scale_pair.restype = C.c_int
         L.mofq_diag_scale_pair.argtypes = [C.c_int, vp, vp, vp, C.c_int64, vp]
         L.mofq_diag_fp_round.restype = C.c_int
@@ -288,6 +290,13 @@ def tensor_error_scaled(x, formats, scales, workspace=None):
     ws = workspace if workspace is not None else _workspace(L.mofq_tensor_workspace_bytes(C.byref(d)), x.device)
     _check(L.mofq_tensor_error_scaled(C.byref(d), fm, n, sc.data_ptr(), out.data_ptr(), ws.data_ptr(), ws.numel(), _stream(x.device)))
     return out, ws[:4].view(torch.int32)
+
+
+def diag_wait_expiry(device):
+    """mofq_diag_wait_expiry: returns a 1-element int32 CUDA tensor that holds MOFQ_STATUS_TIMEOUT once the kernel ends."""
+    out = torch.zeros(1, dtype=torch.int32, device=device)
+    _check(lib().mofq_diag_wait_expiry(out.data_ptr(), _stream(device)))
+    return out
 
 
 def diag_scale_pair(fmt, absmax):

@@ -1,6 +1,7 @@
 // Diagnostic entry point: exposes the grid rounding that the scoring kernels perform with the hardware
 // converts, so that a test can compare it value by value with the definition (nearest grid point, ties to even).
 #include "kq_math.cuh"
+#include "kq_pipe.cuh"
 #include "mofq_internal.h"
 
 namespace {
@@ -23,7 +24,28 @@ __global__ void diag_scale_pair(const float *__restrict__ a, float Q, float rQ, 
     if (i < n) mofq::kqmath::scale_pair_fast(a[i], Q, rQ, s[i], inv[i]);
 }
 
+// waits, with the library's bounded wait, on a barrier that nothing ever arrives on
+__global__ void diag_wait_expiry(int32_t *status_out)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int err;
+    if (threadIdx.x == 0) {
+        mofq::kqpipe::mbar_init(&bar, 1);
+        err = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const bool ok = mofq::kqpipe::mbar_wait(&bar, 0, &err);
+        *status_out = ok ? 0 : MOFQ_STATUS_TIMEOUT;
+    }
+}
+
 }  // namespace
+
+extern "C" int mofq_diag_wait_expiry(int32_t *status_out, void *stream)
+{
+    if (!status_out) return MOFQ_ERR_INVALID_ARG;
+    diag_wait_expiry<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status_out);
+    return cudaGetLastError() == cudaSuccess ? MOFQ_OK : MOFQ_ERR_CUDA;
+}
 
 extern "C" int mofq_diag_scale_pair(int format, const float *absmax, float *scale_out, float *inv_out, int64_t n, void *stream)
 {

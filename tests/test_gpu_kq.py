@@ -422,3 +422,19 @@ def test_codes_only_emission_strided_and_every_fp16_pattern(orc, dev):
     for name in FMT4 + FMT8:
         for gran, group in (("group", 128), ("group", 8), ("tensor", 0)):
             _check_codes_only(orc, x, name, gran, group)
+
+
+def test_bounded_wait_expires_and_leaves_the_context_usable(orc, dev):
+    """A wait that can never be satisfied ends after its limit with a status bit; the GPU stays usable."""
+    import time
+    from paper_2305_12356_b200.binding import diag_wait_expiry
+    t0 = time.time()
+    st = diag_wait_expiry(dev)
+    torch.cuda.synchronize()
+    dt = time.time() - t0
+    assert int(st.item()) == B.STATUS_TIMEOUT
+    assert 0.5 < dt < 10.0, dt                                                    # about two seconds, never a hang
+    x = _weights(dev, 16, 256, seed=61)                                           # and ordinary work still runs
+    got, s2 = mofq.tensor_error(x, ["INT4", "FP4_E2M1"], "channel")
+    want = _oracle_mse(orc, host(x), ["INT4", "FP4_E2M1"], "channel", 0)
+    assert int(s2.item()) == 0 and rel_err(got.cpu().numpy(), want).max() < MSE_RTOL
