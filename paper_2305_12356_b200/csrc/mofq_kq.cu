@@ -221,54 +221,6 @@ __device__ void block_finish(double *acc, int status, WsHeader *hdr, double *par
     }
 }
 
-// ---- scoring kernel 1: dense tensor, per-group scales -------------------------------------------------
-// A tile is 128 consecutive groups staged in shared memory; thread g owns group g and walks its
-// 16-byte chunks in an order rotated by g, which keeps the quarter-warps on distinct banks.
-constexpr int kGroupsPerTile = 128;
-
-template <int DT, int NI, int NFP>
-__global__ void __launch_bounds__(kGroupsPerTile)
-kq_score_groups(const uint16_t *__restrict__ x, long long n_groups, int group, CandSet cs, WsHeader *hdr,
-                double *partials, Finalize fin)
-{
-    constexpr int NC = NI + NFP;
-    extern __shared__ __align__(16) unsigned char smem[];
-    __shared__ double red[33 * NC];
-    const int cpg = group >> 3;  // 16-byte chunks per group (power of two)
-    const long long n_tiles = (n_groups + kGroupsPerTile - 1) / kGroupsPerTile;
-    double dacc[NC];
-#pragma unroll
-    for (int j = 0; j < NC; ++j) dacc[j] = 0.0;
-    int status = 0;
-
-    for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        const long long g0 = tile * kGroupsPerTile;
-        const int ng = (int)min((long long)kGroupsPerTile, n_groups - g0);
-        const int chunks = ng * cpg;
-        const unsigned char *src = reinterpret_cast<const unsigned char *>(x) + (size_t)g0 * group * 2;
-        for (int q = threadIdx.x; q < chunks; q += kGroupsPerTile) cp_async16(smem + q * 16, src + (size_t)q * 16);
-        cp_async_wait_all();
-        __syncthreads();
-        if ((int)threadIdx.x < ng) {
-            const uint4 *base = reinterpret_cast<const uint4 *>(smem) + threadIdx.x * cpg;
-            uint32_t m = 0;
-            for (int j = 0; j < cpg; ++j) m = absmax_chunk(base[(j + threadIdx.x) & (cpg - 1)], m);
-            const uint32_t m16 = fold16(m);
-            if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
-            Scales<NC> sc;
-            make_scales<NI, NFP>(mag16_to_float<DT>(m16), cs, sc, status);
-            float acc[NC];
-#pragma unroll
-            for (int j = 0; j < NC; ++j) acc[j] = 0.0f;
-            for (int j = 0; j < cpg; ++j) score_chunk<DT, NI, NFP>(base[(j + threadIdx.x) & (cpg - 1)], sc, cs, acc);
-#pragma unroll
-            for (int j = 0; j < NC; ++j) dacc[j] += (double)acc[j];
-        }
-        __syncthreads();
-    }
-    block_finish<NC>(dacc, status, hdr, partials, fin, red);
-}
-
 // ---- scoring kernel 2: one row per block; per-channel and/or per-group scales ---------------------------
 // The row is staged in shared memory so that the abs-max pass and the scoring pass cost one HBM read.
 // Work is chunk-strided (a chunk = 8 elements = 16 bytes), so every thread stays busy whatever the row
@@ -474,7 +426,7 @@ kq_select_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long 
                     pick = i;
                 }
             }
-            bs.choice[b] = (uint8_t)pick;
+            if (bs.choice) bs.choice[b] = (uint8_t)pick;
 #pragma unroll
             for (int j = 0; j < NC; ++j) dacc[j] += (double)e[j];
             dacc[NC] += (double)best;
@@ -1305,7 +1257,8 @@ int launch_select_blocks(const ScoreJob &job, uint8_t *choice, float *block_sse,
 {
     const mofq_tensor &x = job.x;
     if (job.gran != MOFQ_PER_CHANNEL && job.gran != MOFQ_PER_GROUP) return MOFQ_ERR_UNSUPPORTED;
-    if (x.cols > 0x7fffffffLL || job.fin.n_cand + 1 > MOFQ_MAX_CAND) return MOFQ_ERR_UNSUPPORTED;
+    const bool with_map = choice != nullptr;   // without a format map this is plain per-block-scale scoring
+    if (x.cols > 0x7fffffffLL || (with_map && job.fin.n_cand + 1 > MOFQ_MAX_CAND)) return MOFQ_ERR_UNSUPPORTED;
     const int width = job.gran == MOFQ_PER_GROUP ? job.group : (int)x.cols;
     const int cpb = width >> 3;
     const int team = (cpb <= 128 && (cpb & (cpb - 1)) == 0) ? std::max(1, cpb / 4) : 32;
@@ -1326,8 +1279,10 @@ int launch_select_blocks(const ScoreJob &job, uint8_t *choice, float *block_sse,
     std::memcpy(bs.perm, job.fin.perm, sizeof(bs.perm));
     // the finalize step reports the candidates in the caller's order and then the mixture (accumulator nc)
     Finalize fin = job.fin;
-    fin.perm[fin.n_cand] = fin.nc;
-    fin.n_cand += 1;
+    if (with_map) {
+        fin.perm[fin.n_cand] = fin.nc;
+        fin.n_cand += 1;
+    }
     fin.nc += 1;
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
 #define MOFQ_BLK(DT_, NI_, K0_, K1_)                                                                              \
@@ -1462,22 +1417,10 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
         });
     }
 
-    if (has_grp && !has_ch && dense) {
-        const long long n_groups = x.rows * x.cols / job.group;
-        const size_t smem = (size_t)kGroupsPerTile * job.group * 2;
-        return dispatch_cands(x.dtype, job.cs.n_int, job.cs.n_fp, [&](auto DT, auto NI, auto NFP) {
-            auto kernel = kq_score_groups<DT(), NI(), NFP()>;
-            if (int rc = set_smem(kernel, smem)) return rc;
-            const int occ = std::max(1, blocks_per_sm((const void *)kernel, kGroupsPerTile, smem));
-            const long long tiles = (n_groups + kGroupsPerTile - 1) / kGroupsPerTile;
-            const int grid = (int)std::min<long long>(tiles, std::min<long long>((long long)nsm * occ, kMaxSlots));
-            kernel<<<grid, kGroupsPerTile, smem, st>>>(xp, n_groups, job.group, job.cs, job.hdr, job.partials, job.fin);
-            MOFQ_CUDA_OK(cudaGetLastError());
-            return MOFQ_OK;
-        });
-    }
+    // group scales only (dense or strided): the register-resident team kernel, without a format map
+    if (has_grp && !has_ch) return launch_select_blocks(job, nullptr, nullptr, st);
 
-    // row kernel: per-channel, per-group on a strided tensor, or both from one read
+    // row kernels: per-channel scales, alone or with group scales from the same read
     if (x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
     if (has_ch && x.cols % 128 == 0 && x.cols * 2 <= kRsMaxTileBytes && (!has_grp || job.group == 128))
         return launch_score_rows_stream(job, has_grp, st);
@@ -1505,8 +1448,7 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
 #define MOFQ_ROWS(DT_, NI_, K0_, K1_)                                                                   \
     if (x.dtype == DT_ && job.cs.n_int == NI_ && k0 == K0_ && k1 == K1_) {                              \
         if (has_ch && has_grp) return launch(kq_score_rows<DT_, NI_, K0_, K1_, true, true>);            \
-        if (has_ch) return launch(kq_score_rows<DT_, NI_, K0_, K1_, true, false>);                      \
-        return launch(kq_score_rows<DT_, NI_, K0_, K1_, false, true>);                                  \
+        return launch(kq_score_rows<DT_, NI_, K0_, K1_, true, false>);                                  \
     }
 #define MOFQ_ROWS_DT(DT_)                                                                                        \
     MOFQ_ROWS(DT_, 1, -1, -1) MOFQ_ROWS(DT_, 0, 0, -1) MOFQ_ROWS(DT_, 1, 0, -1) MOFQ_ROWS(DT_, 0, 0, 0) MOFQ_ROWS(DT_, 1, 0, 0) \

@@ -160,7 +160,7 @@ def test_tensor_error_two_granularities_from_one_read(orc, dev, kind, kw):
         assert rel_err(got.cpu().numpy(), want).max() < MSE_RTOL
 
 
-def test_tensor_error_strided_group_uses_row_kernel(orc, dev):
+def test_tensor_error_strided_group_scales(orc, dev):
     full = _weights(dev, 48, 2048, seed=23)
     view = full[:, 512:1536]
     got, _ = mofq.tensor_error(view, ["INT4", "FP4_E2M1"], "group", group=128)
