@@ -62,19 +62,6 @@ __device__ __forceinline__ void cp_async_wait_all()
     asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
 }
 
-template <int NC>
-struct Scales {
-    float s[NC], inv[NC];
-};
-
-template <int NI, int NFP>
-__device__ __forceinline__ void make_scales(float a, const CandSet &c, Scales<NI + NFP> &sc, int &status)
-{
-    if (NI) scale_pair(a, c.int_q, sc.s[0], sc.inv[0], status);
-#pragma unroll
-    for (int f = 0; f < NFP; ++f) scale_pair(a, c.fp_q[f], sc.s[NI + f], sc.inv[NI + f], status);
-}
-
 // |t| -> nearest FP grid magnitude (RNE), no saturation (|t| <= Q(1+2^-23) under abs-max scales)
 __device__ __forceinline__ float fp_grid_round(float t, uint32_t eminb, uint32_t kadd)
 {
@@ -83,37 +70,6 @@ __device__ __forceinline__ float fp_grid_round(float t, uint32_t eminb, uint32_t
     return __fsub_rn(__fadd_rn(t, c), c);
 }
 
-// one magnitude a = |x| scored against every candidate
-template <int NI, int NFP>
-__device__ __forceinline__ void score1(float a, const Scales<NI + NFP> &sc, const CandSet &c, float *acc)
-{
-    if (NI) {
-        const float t = __fmul_rn(a, sc.inv[0]);
-        const float r = __fsub_rn(__fadd_rn(t, kMagic), kMagic);
-        const float e = __fmaf_rn(-r, sc.s[0], a);
-        acc[0] = __fmaf_rn(e, e, acc[0]);
-    }
-#pragma unroll
-    for (int f = 0; f < NFP; ++f) {
-        const float t = __fmul_rn(a, sc.inv[NI + f]);
-        const float r = fp_grid_round(t, c.fp_eminb[f], c.fp_kadd[f]);
-        const float e = __fmaf_rn(-r, sc.s[NI + f], a);
-        acc[NI + f] = __fmaf_rn(e, e, acc[NI + f]);
-    }
-}
-
-template <int DT, int NI, int NFP>
-__device__ __forceinline__ void score_chunk(const uint4 v, const Scales<NI + NFP> &sc, const CandSet &c, float *acc)
-{
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float lo, hi;
-        unpack2<DT>(w[i], lo, hi);
-        score1<NI, NFP>(fabsf(lo), sc, c, acc);
-        score1<NI, NFP>(fabsf(hi), sc, c, acc);
-    }
-}
 
 // ---- block reductions and the last-block-done finish -------------------------------------------------
 __device__ __forceinline__ uint32_t block_max_u32(uint32_t v, uint32_t *red /* >= 33 words */)
@@ -626,7 +582,19 @@ kq_absmax(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, lo
 {
     uint32_t m = 0;
     const long long total = rows * chunks_per_row;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (rows == 1) {  // dense: no row arithmetic, four independent loads in flight per thread
+        const uint4 *p = reinterpret_cast<const uint4 *>(x);
+        for (; i + 3 * stride < total; i += 4 * stride) {
+            const uint4 v0 = __ldg(p + i), v1 = __ldg(p + i + stride), v2 = __ldg(p + i + 2 * stride), v3 = __ldg(p + i + 3 * stride);
+            m = absmax_chunk(v0, m);
+            m = absmax_chunk(v1, m);
+            m = absmax_chunk(v2, m);
+            m = absmax_chunk(v3, m);
+        }
+    }
+    for (; i < total; i += stride) {
         const long long r = i / chunks_per_row;
         const int c = (int)(i - r * chunks_per_row);
         m = absmax_chunk(__ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c), m);
@@ -637,41 +605,55 @@ kq_absmax(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, lo
     if ((threadIdx.x & 31) == 0 && m16) atomicMax(&hdr->absmax_bits, m16);
 }
 
-template <int DT, int NI, int NFP>
+// The scale pairs are the same for every element, so the packed scorer runs in its scaled form; its binary32 chains
+// are folded into double every 16 chunks (128 terms).
+template <int DT, int NI, int K0, int K1>
 __global__ void __launch_bounds__(256)
-kq_score_uniform(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, CandSet cs,
+kq_score_uniform(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, RowQ rq,
                  WsHeader *hdr, double *partials, Finalize fin)
 {
-    constexpr int NC = NI + NFP;
+    using S = kqmath::Scorer<DT, NI, K0, K1, true>;
+    constexpr int NC = S::NC;
     __shared__ double red[33 * NC];
     int status = 0;
     const uint32_t m16 = *reinterpret_cast<volatile uint32_t *>(&hdr->absmax_bits);
     if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
-    Scales<NC> sc;
-    make_scales<NI, NFP>(mag16_to_float<DT>(m16), cs, sc, status);
+    kqmath::Sc<NC> sc;
+#pragma unroll
+    for (int j = 0; j < NC; ++j) scale_pair(mag16_to_float<DT>(m16), rq.q[j], sc.s[j], sc.inv[j], status);
+    S scorer;
+    scorer.begin(sc);
     double dacc[NC];
 #pragma unroll
     for (int j = 0; j < NC; ++j) dacc[j] = 0.0;
     const long long total = rows * chunks_per_row;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     int n = 0;
-    float acc[NC];
-#pragma unroll
-    for (int j = 0; j < NC; ++j) acc[j] = 0.0f;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    if (rows == 1) {  // dense: no row arithmetic, the next pair of chunks is loaded while this pair is scored
+        const uint4 *p = reinterpret_cast<const uint4 *>(x);
+        for (; i + stride < total; i += 2 * stride) {
+            const uint4 v0 = __ldg(p + i), v1 = __ldg(p + i + stride);
+            scorer.chunk(v0);
+            scorer.chunk(v1);
+            if ((n += 2) >= 16) {
+                scorer.end(dacc);
+                scorer.clear();
+                n = 0;
+            }
+        }
+    }
+    for (; i < total; i += stride) {
         const long long r = i / chunks_per_row;
         const int c = (int)(i - r * chunks_per_row);
-        score_chunk<DT, NI, NFP>(__ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c), sc, cs, acc);
-        if (++n == 16) {  // keep the binary32 chains short: 128 terms, then fold into double
-#pragma unroll
-            for (int j = 0; j < NC; ++j) {
-                dacc[j] += (double)acc[j];
-                acc[j] = 0.0f;
-            }
+        scorer.chunk(__ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c));
+        if (++n >= 16) {
+            scorer.end(dacc);
+            scorer.clear();
             n = 0;
         }
     }
-#pragma unroll
-    for (int j = 0; j < NC; ++j) dacc[j] += (double)acc[j];
+    scorer.end(dacc);
     block_finish<NC>(dacc, status, hdr, partials, fin, red);
 }
 
@@ -1410,11 +1392,28 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
         else
             kq_absmax<1><<<grid, 256, 0, st>>>(xp, rows, (int)cpr, x.ld, job.hdr);
         MOFQ_CUDA_OK(cudaGetLastError());
-        return dispatch_cands(x.dtype, job.cs.n_int, job.cs.n_fp, [&](auto DT, auto NI, auto NFP) {
-            kq_score_uniform<DT(), NI(), NFP()><<<grid, 256, 0, st>>>(xp, rows, (int)cpr, x.ld, job.cs, job.hdr, job.partials, job.fin);
-            MOFQ_CUDA_OK(cudaGetLastError());
-            return MOFQ_OK;
-        });
+        RowQ rq{};
+        if (job.cs.n_int) rq.q[0] = job.cs.int_q;
+        for (int f = 0; f < job.cs.n_fp; ++f) rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
+        auto kind = [](int format) {
+            return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
+        };
+        const int k0 = job.cs.n_fp > 0 ? kind(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? kind(job.fp_formats[1]) : -1;
+#define MOFQ_UNI(DT_, NI_, K0_, K1_)                                                                                      \
+    if (x.dtype == DT_ && job.cs.n_int == NI_ && k0 == K0_ && k1 == K1_) {                                                \
+        kq_score_uniform<DT_, NI_, K0_, K1_><<<grid, 256, 0, st>>>(xp, rows, (int)cpr, x.ld, rq, job.hdr, job.partials, job.fin); \
+        MOFQ_CUDA_OK(cudaGetLastError());                                                                                 \
+        return MOFQ_OK;                                                                                                   \
+    }
+#define MOFQ_UNI_DT(DT_)                                                                                                  \
+    MOFQ_UNI(DT_, 1, -1, -1) MOFQ_UNI(DT_, 0, 0, -1) MOFQ_UNI(DT_, 1, 0, -1) MOFQ_UNI(DT_, 0, 0, 0) MOFQ_UNI(DT_, 1, 0, 0) \
+    MOFQ_UNI(DT_, 0, 1, -1) MOFQ_UNI(DT_, 1, 1, -1) MOFQ_UNI(DT_, 0, 2, -1) MOFQ_UNI(DT_, 1, 2, -1)                     \
+    MOFQ_UNI(DT_, 0, 1, 2) MOFQ_UNI(DT_, 1, 1, 2) MOFQ_UNI(DT_, 0, 2, 1) MOFQ_UNI(DT_, 1, 2, 1)
+        MOFQ_UNI_DT(0)
+        MOFQ_UNI_DT(1)
+#undef MOFQ_UNI_DT
+#undef MOFQ_UNI
+        return MOFQ_ERR_UNSUPPORTED;
     }
 
     // group scales only (dense or strided): the register-resident team kernel, without a format map
