@@ -1137,7 +1137,7 @@ kq_emit_codes_uniform(const uint16_t *__restrict__ x, long long rows, int chunks
     }
     const long long total = rows * chunks_per_row;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-        const long long r = i / chunks_per_row;
+        const long long r = rows == 1 ? 0 : i / chunks_per_row;
         const int c = (int)(i - r * chunks_per_row);
         const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c);
         for (int f = 0; f < es.n; ++f) {
@@ -1478,10 +1478,14 @@ int launch_emit_codes_uniform(const mofq_tensor &x, int n, const int *formats, v
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
     const long long total = x.rows * (x.cols / 8);
     const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
+    // a dense tensor is one long row for this kernel (the codes are dense either way): no per-chunk row arithmetic
+    const bool flat = x.ld == x.cols && total <= 0x7fffffffLL;
+    const long long rows = flat ? 1 : x.rows;
+    const int cpr = flat ? (int)total : (int)(x.cols / 8);
     if (x.dtype == MOFQ_F16)
-        kq_emit_codes_uniform<0><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, es, hdr);
+        kq_emit_codes_uniform<0><<<grid, 256, 0, st>>>(xp, rows, cpr, x.ld, es, hdr);
     else
-        kq_emit_codes_uniform<1><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, es, hdr);
+        kq_emit_codes_uniform<1><<<grid, 256, 0, st>>>(xp, rows, cpr, x.ld, es, hdr);
     MOFQ_CUDA_OK(cudaGetLastError());
     return MOFQ_OK;
 }
