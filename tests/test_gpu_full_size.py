@@ -116,3 +116,25 @@ def test_large_single_tensor_group_scales_takes_the_streaming_route(orc, dev):
     w[7000, 123] = float("inf")
     _, st = mofq.tensor_error(w, names, "group", group=128)
     assert int(st.item()) & mofq.binding.STATUS_NONFINITE_INPUT
+
+
+def test_tensor_beyond_2_to_31_elements_splits_consistently(dev):
+    """Index arithmetic past 2^31 elements: a 65536 x 65536 tensor (8.6 GB) scored whole equals its halves combined."""
+    w = torch.empty((65536, 65536), dtype=torch.float16, device=dev)
+    for q in range(4):                                                     # four seeded quarters (the generator is per call)
+        inputs.device_weight(w[q * 16384:(q + 1) * 16384], "student_t", 9, q)
+    names = ["INT4", "FP4_E2M1"]
+    for gran, group in (("group", 128), ("channel", 0)):
+        whole, st = mofq.tensor_error(w, names, gran, group=group)
+        top, _ = mofq.tensor_error(w[:32768], names, gran, group=group)
+        bot, _ = mofq.tensor_error(w[32768:], names, gran, group=group)
+        assert int(st.item()) == 0
+        both = (top.double() + bot.double()) / 2
+        assert rel_err(whole.cpu().numpy(), both.cpu().numpy()).max() < MSE_RTOL, (gran, whole, both)
+    got = mofq.quantize_tensor(w, "FP4_E2M1", "group", 128, want_scales=True)
+    part = mofq.quantize_tensor(w[65000:], "FP4_E2M1", "group", 128)       # the tail rows, quantised on their own
+    n_tail = (65536 - 65000) * 65536
+    assert torch.equal(got["codes"][-n_tail // 2:], part["codes"])
+    assert torch.equal(got["scales"][-n_tail // 128:], part["scales"])
+    del w, got, part
+    torch.cuda.empty_cache()
