@@ -198,25 +198,29 @@ __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr)
            (2ull << 61) /* 128-byte swizzle */;
 }
 
+constexpr int kMaxProb = 3;     // products of one shape that one launch can carry (the candidates of a layer)
 struct GemmParams {
     int M, N, K;              // Y is M x N, contraction over K
     int mode;                 // 0: reference (write Y, sum Y^2); 1: quantised (sum (Y - alpha*col*acc)^2)
+    int n_prob;               // products in this launch; their tiles form one list, so the waves are shared
     float *Y;                 // [M, N] fp32, dense
-    const float *alpha;       // device scalar
-    const float *col_scale;   // device [N] or nullptr (treated as 1)
-    double *partials;         // one double per CTA
+    const float *alpha[kMaxProb];      // device scalar per product
+    const float *col_scale[kMaxProb];  // device [N] or nullptr (treated as 1)
+    double *partials[kMaxProb];        // one double per CTA and product
     int32_t *status;          // device status word (timeout)
-    uint32_t idesc;
-    int kind;                 // operand kind of the MMA: KIND_F16 (fp16/bf16), KIND_I8 (int8 -> int32), KIND_F8 (e4m3/e5m2)
-    int bk;                   // elements of K per tile row (64 or 128)
+    uint32_t idesc[kMaxProb];
+    int kind[kMaxProb];       // operand kind of the MMA: KIND_F16 (fp16/bf16), KIND_I8 (int8 -> int32), KIND_F8 (e4m3/e5m2)
+    int bk;                   // elements of K per tile row (64 or 128), the same for every product of a launch
     int y_tma;                // mode 0: Y is written by TMA stores through map_y
+};
+struct GemmMaps {             // operand tensor maps of the products
+    CUtensorMap a[kMaxProb], b[kMaxProb];
 };
 enum { KIND_F16 = 0, KIND_I8 = 1, KIND_F8 = 2 };
 
 template <int BN, int CG>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const __grid_constant__ CUtensorMap map_y, const GemmParams p)
+gemm_err_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ CUtensorMap map_y, const GemmParams p)
 {
     using Cfg = TileCfg<BN, CG>;
     constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes, kTmemCols = Cfg::kTmemCols;
@@ -224,7 +228,7 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], tfull_bar[2], tempty_bar[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int err_flag;
-    __shared__ double red[kEpiWarps];
+    __shared__ double red[kEpiWarps][kMaxProb];
     volatile int *const perr = &err_flag;
 #define err (*perr)
 
@@ -233,7 +237,8 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int rank = CG == 2 ? (int)cluster_ctarank() : 0;            // 0 = leader of the pair
     const int unit = (int)blockIdx.x / CG, n_units = (int)gridDim.x / CG;  // a unit (CTA or pair) owns whole tiles
     const int tiles_m = (p.M + BM * CG - 1) / (BM * CG), tiles_n = (p.N + BN - 1) / BN;
-    const int n_tiles = tiles_m * tiles_n;
+    const int n_tiles = tiles_m * tiles_n;          // per product
+    const int all_tiles = n_tiles * p.n_prob;       // the launch's tile list: product-major
     constexpr int KA = Cfg::KA;
     const int kblocks = (p.K + p.bk * KA - 1) / (p.bk * KA);  // a k-block is one stage: KA atoms of K
 
@@ -247,7 +252,8 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             mbar_init(&tempty_bar[b], kEpiWarps * CG);  // the epilogue warps of every CTA of the unit release the leader
         }
         err = 0;
-        for (int i = 0; i < kEpiWarps; ++i) red[i] = 0.0;
+        for (int i = 0; i < kEpiWarps; ++i)
+            for (int j = 0; j < kMaxProb; ++j) red[i][j] = 0.0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // the MMA warp owns the tensor-memory allocation
@@ -269,7 +275,9 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             int it = 0;
-            for (int tile = unit; tile < n_tiles && !err; tile += n_units) {
+            for (int gt = unit; gt < all_tiles && !err; gt += n_units) {
+                const int prob = gt / n_tiles, tile = gt - prob * n_tiles;
+                const CUtensorMap *map_a = &maps.a[prob], *map_b = &maps.b[prob];
                 // m fastest: co-running tiles share a B tile.  This CTA's rows of A and of B inside the unit's tile:
                 const int m0 = (tile % tiles_m) * BM * CG + rank * BM, n0 = (tile / tiles_m) * BN + rank * Cfg::kBRows;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -282,15 +290,15 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         const uint32_t leader_bar = mapa_u32(smem_u32(&full_bar[s]), 0);
 #pragma unroll
                         for (int a = 0; a < KA; ++a) {
-                            tma_load_2d_pair(st + a * kABytes, &map_a, (kb * KA + a) * p.bk, m0, leader_bar);
-                            tma_load_2d_pair(st + KA * kABytes + a * Cfg::kBBytes, &map_b, (kb * KA + a) * p.bk, n0, leader_bar);
+                            tma_load_2d_pair(st + a * kABytes, map_a, (kb * KA + a) * p.bk, m0, leader_bar);
+                            tma_load_2d_pair(st + KA * kABytes + a * Cfg::kBBytes, map_b, (kb * KA + a) * p.bk, n0, leader_bar);
                         }
                     } else {
                         mbar_expect_tx(&full_bar[s], kStageBytes);
 #pragma unroll
                         for (int a = 0; a < KA; ++a) {
-                            tma_load_2d(st + a * kABytes, &map_a, (kb * KA + a) * p.bk, m0, &full_bar[s]);
-                            tma_load_2d(st + KA * kABytes + a * Cfg::kBBytes, &map_b, (kb * KA + a) * p.bk, n0, &full_bar[s]);
+                            tma_load_2d(st + a * kABytes, map_a, (kb * KA + a) * p.bk, m0, &full_bar[s]);
+                            tma_load_2d(st + KA * kABytes + a * Cfg::kBBytes, map_b, (kb * KA + a) * p.bk, n0, &full_bar[s]);
                         }
                     }
                 }
@@ -307,54 +315,60 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // The tensor pipe takes an MMA only when it can start it, so whatever else this thread does between MMAs is
         // a bubble: the loop is kept to a barrier wait, KA*4 MMAs whose descriptors are one 64-bit add away, a commit.
         if (lane == 0 && rank == 0) {
-            const uint32_t idesc = p.idesc;
             const uint64_t a_desc0 = smem_desc_k_major_sw128(smem_u32(smem));
             const uint64_t b_desc0 = smem_desc_k_major_sw128(smem_u32(smem + KA * kABytes));
-            auto run = [&](auto kind_tag) {
+            int s = 0;
+            uint32_t ph = 0;
+            uint64_t a_desc = a_desc0, b_desc = b_desc0;  // descriptors of the current stage (address field in 16-byte units)
+            // the main loop of one tile for one operand kind; false = a bounded wait expired
+            auto tile_mmas = [&](auto kind_tag, uint32_t idesc, uint32_t d_tmem) -> bool {
                 constexpr int KIND = decltype(kind_tag)::value;
-                int s = 0, local = 0;
-                uint32_t ph = 0;
-                uint64_t a_desc = a_desc0, b_desc = b_desc0;  // descriptors of the current stage (address field in 16-byte units)
-                for (int tile = unit; tile < n_tiles && !err; tile += n_units, ++local) {
-                    const int buf = local & 1;
-                    if (!mbar_wait(&tempty_bar[buf], ((local >> 1) & 1) ^ 1, perr)) return;
-                    tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                    uint32_t acc = 0;
-                    for (int kb = 0; kb < kblocks; ++kb) {
-                        // (no tcgen05 fence here: the mbarrier orders the TMA data for the MMAs)
-                        if (!mbar_wait(&full_bar[s], ph, perr)) return;
+                uint32_t acc = 0;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    // (no tcgen05 fence here: the mbarrier orders the TMA data for the MMAs)
+                    if (!mbar_wait(&full_bar[s], ph, perr)) return false;
 #pragma unroll
-                        for (int k = 0; k < KA * (kRowBytes / 32); ++k) {  // one MMA consumes 32 bytes of K
-                            constexpr int per = kRowBytes / 32;
-                            const uint64_t ad = a_desc + (uint64_t)((k / per) * (kABytes >> 4) + 2 * (k % per));
-                            const uint64_t bd = b_desc + (uint64_t)((k / per) * (Cfg::kBBytes >> 4) + 2 * (k % per));
-                            if (CG == 2) tc_mma_pair<KIND>(d_tmem, ad, bd, idesc, acc);
-                            else if (KIND == KIND_F16) tc_mma_f16(d_tmem, ad, bd, idesc, acc);
-                            else if (KIND == KIND_I8) tc_mma_i8(d_tmem, ad, bd, idesc, acc);
-                            else tc_mma_f8(d_tmem, ad, bd, idesc, acc);
-                            acc = 1;
-                        }
-                        // the stage is free (in every CTA of the unit) once these MMAs have read it
-                        if (CG == 2) tc_commit_pair(&empty_bar[s]);
-                        else tc_commit(&empty_bar[s]);
-                        if (++s == kStages) {
-                            s = 0;
-                            ph ^= 1u;
-                            a_desc = a_desc0;
-                            b_desc = b_desc0;
-                        } else {
-                            a_desc += (uint64_t)(kStageBytes >> 4);
-                            b_desc += (uint64_t)(kStageBytes >> 4);
-                        }
+                    for (int k = 0; k < KA * (kRowBytes / 32); ++k) {  // one MMA consumes 32 bytes of K
+                        constexpr int per = kRowBytes / 32;
+                        const uint64_t ad = a_desc + (uint64_t)((k / per) * (kABytes >> 4) + 2 * (k % per));
+                        const uint64_t bd = b_desc + (uint64_t)((k / per) * (Cfg::kBBytes >> 4) + 2 * (k % per));
+                        if (CG == 2) tc_mma_pair<KIND>(d_tmem, ad, bd, idesc, acc);
+                        else if (KIND == KIND_F16) tc_mma_f16(d_tmem, ad, bd, idesc, acc);
+                        else if (KIND == KIND_I8) tc_mma_i8(d_tmem, ad, bd, idesc, acc);
+                        else tc_mma_f8(d_tmem, ad, bd, idesc, acc);
+                        acc = 1;
                     }
-                    if (CG == 2) tc_commit_pair(&tfull_bar[buf]);  // accumulator complete
-                    else tc_commit(&tfull_bar[buf]);
+                    // the stage is free (in every CTA of the unit) once these MMAs have read it
+                    if (CG == 2) tc_commit_pair(&empty_bar[s]);
+                    else tc_commit(&empty_bar[s]);
+                    if (++s == kStages) {
+                        s = 0;
+                        ph ^= 1u;
+                        a_desc = a_desc0;
+                        b_desc = b_desc0;
+                    } else {
+                        a_desc += (uint64_t)(kStageBytes >> 4);
+                        b_desc += (uint64_t)(kStageBytes >> 4);
+                    }
                 }
+                return true;
             };
-            if (p.kind == KIND_F16) run(std::integral_constant<int, KIND_F16>());
-            else if (p.kind == KIND_I8) run(std::integral_constant<int, KIND_I8>());
-            else run(std::integral_constant<int, KIND_F8>());
+            int local = 0;
+            for (int gt = unit; gt < all_tiles && !err; gt += n_units, ++local) {
+                const int prob = gt / n_tiles;
+                const int buf = local & 1;
+                if (!mbar_wait(&tempty_bar[buf], ((local >> 1) & 1) ^ 1, perr)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                const uint32_t idesc = p.idesc[prob];
+                const int kind = p.kind[prob];
+                const bool ok = kind == KIND_F16  ? tile_mmas(std::integral_constant<int, KIND_F16>(), idesc, d_tmem)
+                                : kind == KIND_I8 ? tile_mmas(std::integral_constant<int, KIND_I8>(), idesc, d_tmem)
+                                                  : tile_mmas(std::integral_constant<int, KIND_F8>(), idesc, d_tmem);
+                if (!ok) break;
+                if (CG == 2) tc_commit_pair(&tfull_bar[buf]);  // accumulator complete
+                else tc_commit(&tfull_bar[buf]);
+            }
         }
     } else {
         // ---------------- epilogue: warps 2..5 read the lane quarter (warp % 4) of the accumulator ----------------
@@ -364,10 +378,13 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int half = (warp - 2) >> 2;                 // which half of the tile's columns this warp handles
         constexpr int kChunks = BN / 32 / (kEpiWarps / 4);
         const uint32_t stage = smem_u32(smem + kRingBytes + (warp - 2) * kStageTile);
-        const float alpha = *p.alpha;
-        double dsum = 0.0;
+        double dsum0 = 0.0, dsum1 = 0.0, dsum2 = 0.0;    // one running sum per product
         int local = 0;
-        for (int tile = unit; tile < n_tiles; tile += n_units, ++local) {
+        for (int gt = unit; gt < all_tiles; gt += n_units, ++local) {
+            const int prob = gt / n_tiles, tile = gt - prob * n_tiles;
+            const float alpha = __ldg(p.alpha[prob]);
+            const float *col_scale = p.col_scale[prob];
+            const int kind = p.kind[prob];
             const int buf = local & 1;
             const int m0 = (tile % tiles_m) * BM * CG + rank * BM, n0 = (tile / tiles_m) * BN;
             const int row = m0 + q * 32 + lane;
@@ -400,7 +417,7 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 tc_ld_wait(r);
                 if (ci + 1 < kChunks) tc_ld_32x32(t0 + (uint32_t)((c + 1) * 32), rn);
                 const int col0 = n0 + c * 32;
-                if (p.kind == KIND_I8) {  // exact integer dot products -> float
+                if (kind == KIND_I8) {  // exact integer dot products -> float
 #pragma unroll
                     for (int j = 0; j < 32; ++j) r[j] = __float_as_uint((float)(int)r[j]);
                 }
@@ -447,7 +464,7 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                             } else {
                                 const float4 y = ycur[j >> 2];
                                 float4 cs = make_float4(1.f, 1.f, 1.f, 1.f);
-                                if (p.col_scale) cs = __ldg(reinterpret_cast<const float4 *>(p.col_scale + col0 + j));
+                                if (col_scale) cs = __ldg(reinterpret_cast<const float4 *>(col_scale + col0 + j));
                                 const float d0 = y.x - __uint_as_float(r[j]) * (alpha * cs.x);
                                 const float d1 = y.y - __uint_as_float(r[j + 1]) * (alpha * cs.y);
                                 const float d2 = y.z - __uint_as_float(r[j + 2]) * (alpha * cs.z);
@@ -468,7 +485,7 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                                 yrow[j] = v;
                                 fsum = fmaf(v, v, fsum);
                             } else {
-                                const float cs = p.col_scale ? p.col_scale[col0 + j] : 1.0f;
+                                const float cs = col_scale ? col_scale[col0 + j] : 1.0f;
                                 const float d = yrow[j] - a * (alpha * cs);
                                 fsum = fmaf(d, d, fsum);
                             }
@@ -478,7 +495,9 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 8; ++j) ycur[j] = ynext[j];
             }
-            dsum += (double)fsum;
+            if (prob == 0) dsum0 += (double)fsum;
+            else if (prob == 1) dsum1 += (double)fsum;
+            else dsum2 += (double)fsum;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
@@ -488,16 +507,26 @@ gemm_err_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
         if (p.mode == 0 && p.y_tma && lane == 0) tma_store_wait_all();   // Y is in global memory before the block leaves
 #pragma unroll
-        for (int o = 16; o; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
-        if (lane == 0) red[warp - 2] = dsum;
+        for (int o = 16; o; o >>= 1) {
+            dsum0 += __shfl_xor_sync(0xffffffffu, dsum0, o);
+            dsum1 += __shfl_xor_sync(0xffffffffu, dsum1, o);
+            dsum2 += __shfl_xor_sync(0xffffffffu, dsum2, o);
+        }
+        if (lane == 0) {
+            red[warp - 2][0] = dsum0;
+            red[warp - 2][1] = dsum1;
+            red[warp - 2][2] = dsum2;
+        }
     }
     tc_fence_before();
     if (CG == 2) cluster_sync();  // no CTA leaves while its peer may still touch its shared or tensor memory
     else __syncthreads();
     if (threadIdx.x == 0) {
-        double tot = 0.0;
-        for (int i = 0; i < kEpiWarps; ++i) tot += red[i];
-        p.partials[blockIdx.x] = tot;
+        for (int j = 0; j < p.n_prob; ++j) {
+            double tot = 0.0;
+            for (int i = 0; i < kEpiWarps; ++i) tot += red[i][j];
+            p.partials[j][blockIdx.x] = tot;
+        }
         if (err) atomicOr(p.status, MOFQ_STATUS_TIMEOUT);
     }
     if (warp == 1) {
@@ -540,7 +569,8 @@ __global__ void set_scalar(float *p, float v) { *p = v; }
 
 struct LayerFinalize {
     const double *partials;  // [(1 + n_cand)][stride]
-    int stride, n_ctas, n_cand;
+    int stride, n_cand;
+    int n_ctas[1 + MOFQ_MAX_CAND];  // blocks that wrote each entry's partial sums (launch grids can differ)
     double inv_n;
     mofq_result *res;
     float *mse_out, *nsr_out;
@@ -553,7 +583,7 @@ layer_finalize(const LayerFinalize f)
     double tot[1 + MOFQ_MAX_CAND];
     for (int k = 0; k <= f.n_cand; ++k) {
         double s = 0.0;
-        for (int c = threadIdx.x; c < f.n_ctas; c += 32) s += f.partials[(size_t)k * f.stride + c];
+        for (int c = threadIdx.x; c < f.n_ctas[k]; c += 32) s += f.partials[(size_t)k * f.stride + c];
 #pragma unroll
         for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         tot[k] = s;
@@ -650,48 +680,57 @@ LayerWs layer_ws_layout(long long T, long long n_in, long long n_out)
 
 // op: MOFQ_F16 / MOFQ_BF16 (16-bit operands), or an 8-bit mofq_format (MOFQ_INT8, MOFQ_FP8_E4M3, MOFQ_FP8_E5M2) + 100
 constexpr int kOp8 = 100;
-int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, long long b_rows, long long b_ld, long long K,
-             int op, int mode, float *Y, const float *alpha, const float *col_scale, double *partials, int32_t *status,
-             int *grid_out, cudaStream_t st)
+// One launch over n products of the same shape (the candidates of a layer): their tiles form one list, so the last
+// wave is shared instead of paid once per product.  n = 1 for the reference pass.
+int run_gemm_n(int n, const void *const *a, long long a_rows, const long long *a_ld, const void *const *b, long long b_rows,
+               long long b_ld, long long K, const int *op, int mode, float *Y, const float *const *alpha,
+               const float *const *col_scale, double *const *partials, int32_t *status, int *grid_out, cudaStream_t st)
 {
+    if (n < 1 || n > kMaxProb) return MOFQ_ERR_INVALID_ARG;
     // tile shape: waves x relative tile cost.  Operand bytes per CTA and k-block: 32 KB for a 128x128 tile, 48 KB for
     // 128x256, and 32 KB per CTA for a CTA pair sharing a 256x256 tile (cost per 128x128 of output: 1, 0.75, 0.5).
     const int nsm = sm_count();
     const long long mt = (a_rows + BM - 1) / BM;
-    const long long t128 = mt * ((b_rows + 127) / 128), t256 = mt * ((b_rows + 255) / 256);
-    const long long tpair = ((a_rows + 2 * BM - 1) / (2 * BM)) * ((b_rows + 255) / 256);
+    const long long t128 = n * mt * ((b_rows + 127) / 128), t256 = n * mt * ((b_rows + 255) / 256);
+    const long long tpair = n * ((a_rows + 2 * BM - 1) / (2 * BM)) * ((b_rows + 255) / 256);
     const int npair = std::max(1, nsm / 2);
     const double c128 = (double)((t128 + nsm - 1) / nsm) * 1.0, c256 = (double)((t256 + nsm - 1) / nsm) * 1.5;
     const double cpair = (double)((tpair + npair - 1) / npair) * 1.0;
     const bool force_single = getenv("MOFQ_GEMM_SINGLE_CTA") != nullptr;
     const int cg = (!force_single && cpair < std::min(c128, c256)) ? 2 : 1;
     const int bn = cg == 2 ? 256 : (c256 < c128 ? 256 : 128);
-    CUtensorMap map_a, map_b;
-    const int elem = op >= kOp8 ? kElemU8 : op;
-    if (int rc = make_map(&map_a, a, elem, a_rows, K, a_ld, BM)) return rc;
-    if (int rc = make_map(&map_b, b, elem, b_rows, K, b_ld, bn / cg)) return rc;
+    GemmMaps maps;
     GemmParams p{};
+    p.n_prob = n;
+    for (int i = 0; i < kMaxProb; ++i) {
+        const int j = i < n ? i : 0;  // unused slots repeat product 0 so that every map is a valid object
+        const int elem = op[j] >= kOp8 ? kElemU8 : op[j];
+        if ((op[j] >= kOp8) != (op[0] >= kOp8)) return MOFQ_ERR_INVALID_ARG;  // one K-atom width per launch
+        if (int rc = make_map(&maps.a[i], a[j], elem, a_rows, K, a_ld[j], BM)) return rc;
+        if (int rc = make_map(&maps.b[i], b[j], elem, b_rows, K, b_ld, bn / cg)) return rc;
+        p.alpha[i] = alpha[j];
+        p.col_scale[i] = col_scale[j];
+        p.partials[i] = partials[j];
+        // instruction descriptor: accumulator type [4,6), A type [7,10), B type [10,13), both K-major, N/8 at [17,23), M/16 at [24,29)
+        uint32_t cfmt, abfmt;
+        if (op[j] == kOp8 + MOFQ_INT8) {
+            p.kind[i] = KIND_I8; cfmt = 2u /* s32 */; abfmt = 1u /* signed 8-bit */;
+        } else if (op[j] >= kOp8) {
+            p.kind[i] = KIND_F8; cfmt = 1u /* f32 */; abfmt = op[j] == kOp8 + MOFQ_FP8_E4M3 ? 0u : 1u /* e4m3 : e5m2 */;
+        } else {
+            p.kind[i] = KIND_F16; cfmt = 1u; abfmt = op[j] == MOFQ_F16 ? 0u : 1u /* f16 : bf16 */;
+        }
+        p.idesc[i] = (cfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((BM * cg) >> 4) << 24);
+    }
+    const CUtensorMap &map_a = maps.a[0];
     p.M = (int)a_rows;
     p.N = (int)b_rows;
     p.K = (int)K;
     p.mode = mode;
     p.Y = Y;
-    p.alpha = alpha;
-    p.col_scale = col_scale;
-    p.partials = partials;
     p.status = status;
-    // instruction descriptor: accumulator type [4,6), A type [7,10), B type [10,13), both K-major, N/8 at [17,23), M/16 at [24,29)
-    uint32_t cfmt, abfmt;
-    if (op == kOp8 + MOFQ_INT8) {
-        p.kind = KIND_I8; cfmt = 2u /* s32 */; abfmt = 1u /* signed 8-bit */;
-    } else if (op >= kOp8) {
-        p.kind = KIND_F8; cfmt = 1u /* f32 */; abfmt = op == kOp8 + MOFQ_FP8_E4M3 ? 0u : 1u /* e4m3 : e5m2 */;
-    } else {
-        p.kind = KIND_F16; cfmt = 1u; abfmt = op == MOFQ_F16 ? 0u : 1u /* f16 : bf16 */;
-    }
-    p.bk = op >= kOp8 ? kRowBytes : kRowBytes / 2;
-    p.idesc = (cfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((BM * cg) >> 4) << 24);
-    const int tiles = cg == 2 ? (int)tpair : (int)(((a_rows + BM - 1) / BM) * ((b_rows + bn - 1) / bn));
+    p.bk = op[0] >= kOp8 ? kRowBytes : kRowBytes / 2;
+    const int tiles = cg == 2 ? (int)tpair : (int)(n * ((a_rows + BM - 1) / BM) * ((b_rows + bn - 1) / bn));
     const int grid = cg * std::min(tiles, std::min(nsm, kMaxGemmCtas) / cg);
     // the staging tiles are only needed (and only touched) by the reference pass; the candidate passes keep the
     // smaller request so that more of the SM's unified memory stays level-1 cache for their reads of Y
@@ -728,7 +767,7 @@ int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, lon
         attr[0].val.clusterDim.z = 1;
         lc.attrs = attr;
         lc.numAttrs = 1;
-        if (cudaLaunchKernelEx(&lc, kernel, map_a, map_b, map_y, p) != cudaSuccess) {
+        if (cudaLaunchKernelEx(&lc, kernel, maps, map_y, p) != cudaSuccess) {
             (void)cudaGetLastError();
             return MOFQ_ERR_CUDA;
         }
@@ -739,6 +778,13 @@ int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, lon
         return rc;
     *grid_out = grid;
     return MOFQ_OK;
+}
+
+int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, long long b_rows, long long b_ld, long long K,
+             int op, int mode, float *Y, const float *alpha, const float *col_scale, double *partials, int32_t *status,
+             int *grid_out, cudaStream_t st)
+{
+    return run_gemm_n(1, &a, a_rows, &a_ld, &b, b_rows, b_ld, K, &op, mode, Y, &alpha, &col_scale, &partials, status, grid_out, st);
 }
 
 }  // namespace
@@ -819,10 +865,33 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
         }
         if (int rc = launch_emit_codes_uniform(X, cfg->n_candidates, fmts, cptr, sptr, hdr, st)) return rc;
     }
-    int grid_used = 0, max_grid = 0;
+    int grid_used = 0;
+    int grids[1 + MOFQ_MAX_CAND] = {0};
     if (int rc = run_gemm(xa, T, xa_ld, W.data, n_out, W.ld, n_in, op_dtype, 0, Y, scal, nullptr, partials, &hdr->status, &grid_used, st))
         return rc;
-    max_grid = grid_used;
+    grids[0] = grid_used;
+    if (fused && cfg->n_candidates <= kMaxProb) {
+        // every candidate's operands exist already: one launch carries all their products (Algorithm 1's loop over the
+        // formats becomes the product index of the tile list), so the partly filled last wave is paid once
+        const void *ga[kMaxProb], *gb[kMaxProb];
+        long long gld[kMaxProb];
+        int gop[kMaxProb];
+        const float *galpha[kMaxProb], *gcs[kMaxProb];
+        double *gpart[kMaxProb];
+        for (int i = 0; i < cfg->n_candidates; ++i) {
+            ga[i] = reinterpret_cast<unsigned char *>(cx) + (size_t)i * cx_stride;
+            gb[i] = reinterpret_cast<unsigned char *>(cw) + (size_t)i * cw_stride;
+            gld[i] = n_in;
+            gop[i] = kOp8 + cfg->candidates[i];
+            galpha[i] = scal + 1 + i;
+            gcs[i] = sw + (size_t)i * sw_stride;
+            gpart[i] = partials + (size_t)(1 + i) * kMaxGemmCtas;
+        }
+        if (int rc = run_gemm_n(cfg->n_candidates, ga, T, gld, gb, n_out, n_in, n_in, gop, 1, Y, galpha, gcs, gpart, &hdr->status,
+                                &grid_used, st))
+            return rc;
+        for (int i = 0; i < cfg->n_candidates; ++i) grids[1 + i] = grid_used;
+    } else {
     for (int i = 0; i < cfg->n_candidates; ++i) {  // Algorithm 1: for format in format_candidates
         const void *bw = cw;
         const float *bsw = sw;
@@ -851,12 +920,13 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
         if (int rc = run_gemm(a, T, a_ld, bw, n_out, n_in, n_in, op, 1, Y, alpha, bsw, partials + (size_t)(1 + i) * kMaxGemmCtas,
                               &hdr->status, &grid_used, st))
             return rc;
-        max_grid = std::max(max_grid, grid_used);
+        grids[1 + i] = grid_used;
+    }
     }
     LayerFinalize f{};
     f.partials = partials;
     f.stride = kMaxGemmCtas;
-    f.n_ctas = max_grid;
+    for (int k = 0; k <= cfg->n_candidates; ++k) f.n_ctas[k] = grids[k];
     f.n_cand = cfg->n_candidates;
     f.inv_n = 1.0 / ((double)T * (double)n_out);
     f.res = res;
