@@ -361,10 +361,11 @@ def main():
         # algorithmic bytes: 2 B per element read once (+ 4 B per 128 elements of scale state never leaves the SM)
         F = cfg.n_candidates
         flops = sum(2.0 * T * o * i * (1 + F) for _, o, i in shapes) if layer_metric else 0.0
-        # kernels per step, counted from the launch lists in profiles/: layer-output path = (1 + F) GEMMs + abs-max,
+        # kernels per step, counted from the launch lists in profiles/: layer-output path = GEMM launches + abs-max,
         # operand conversion, two code-emission kernels and the finalize per layer; multi-tensor path = table uploads
         # (64 layers each) + the persistent kernel + the finalize; otherwise one scoring kernel per layer
-        launches_per_step = len(shapes) * ((1 + F) + 5) if layer_metric else (2 + (len(shapes) + 63) // 64 if grans == ("group",) else len(shapes))
+        gemm_launches = 2 if (layer_metric and wl["bits"] == 8) else 1 + F   # 8-bit W+A: the candidates share one launch
+        launches_per_step = len(shapes) * (gemm_launches + 5) if layer_metric else (2 + (len(shapes) + 63) // 64 if grans == ("group",) else len(shapes))
         mt = grans == ("group",)
         dom_launches = 1 if mt else len(shapes)      # launches of the dominant kernel per step
         roofline = {"bound": "hbm", "kernel": "kq_score_mt" if mt else "kq_score_rows_stream", "achieved": fp16_bytes / (ms_per_step * 1e-3) / 1e9,
