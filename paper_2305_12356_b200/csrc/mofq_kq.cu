@@ -1171,6 +1171,41 @@ int dispatch_cands(int dt, int ni, int nfp, F &&f)
     return MOFQ_ERR_UNSUPPORTED;
 }
 
+// Canonical candidate set -> compile-time (dtype, INT present, FP kind of slot 0, FP kind of slot 1); kinds are
+// kqmath::FPK_* or -1.  Only the combinations one bit-width allows exist.
+template <typename F>
+int dispatch_kinds(int dt, int ni, int k0, int k1, F &&f)
+{
+#define MOFQ_KIND(DT_, NI_, K0_, K1_)                                                                    \
+    if (dt == DT_ && ni == NI_ && k0 == K0_ && k1 == K1_)                                                \
+        return f(std::integral_constant<int, DT_>(), std::integral_constant<int, NI_>(), std::integral_constant<int, K0_>(), \
+                 std::integral_constant<int, K1_>());
+#define MOFQ_KIND_DT(DT_)                                                                                             \
+    MOFQ_KIND(DT_, 1, -1, -1) MOFQ_KIND(DT_, 0, 0, -1) MOFQ_KIND(DT_, 1, 0, -1) MOFQ_KIND(DT_, 0, 0, 0) MOFQ_KIND(DT_, 1, 0, 0) \
+    MOFQ_KIND(DT_, 0, 1, -1) MOFQ_KIND(DT_, 1, 1, -1) MOFQ_KIND(DT_, 0, 2, -1) MOFQ_KIND(DT_, 1, 2, -1)                         \
+    MOFQ_KIND(DT_, 0, 1, 2) MOFQ_KIND(DT_, 1, 1, 2) MOFQ_KIND(DT_, 0, 2, 1) MOFQ_KIND(DT_, 1, 2, 1)
+    MOFQ_KIND_DT(0)
+    MOFQ_KIND_DT(1)
+#undef MOFQ_KIND_DT
+#undef MOFQ_KIND
+    return MOFQ_ERR_UNSUPPORTED;
+}
+
+int fp_kind_of(int format)
+{
+    return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
+}
+
+// abs-max targets (and their reciprocals) of a job's canonical slots
+RowQ job_rowq(const ScoreJob &job)
+{
+    RowQ rq{};
+    if (job.cs.n_int) rq.q[0] = job.cs.int_q;
+    for (int f = 0; f < job.cs.n_fp; ++f) rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
+    for (int j = 0; j < 3; ++j) rq.rq[j] = rq.q[j] > 0.0f ? 1.0f / rq.q[j] : 0.0f;
+    return rq;
+}
+
 int blocks_per_sm(const void *kernel, int threads, size_t smem)
 {
     int n = 0;
@@ -1247,13 +1282,8 @@ int launch_select_blocks(const ScoreJob &job, uint8_t *choice, float *block_sse,
     const long long n_blocks = x.rows * (x.cols / width);
     const long long warps = (n_blocks + (32 / team) - 1) / (32 / team);
     const int grid = (int)std::min<long long>((warps + 7) / 8, std::min<long long>((long long)sm_count() * 8, kMaxSlots));
-    RowQ rq{};
-    if (job.cs.n_int) rq.q[0] = job.cs.int_q;
-    for (int f = 0; f < job.cs.n_fp; ++f) rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
-    auto kind = [](int format) {
-        return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
-    };
-    const int k0 = job.cs.n_fp > 0 ? kind(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? kind(job.fp_formats[1]) : -1;
+    const RowQ rq = job_rowq(job);
+    const int k0 = job.cs.n_fp > 0 ? fp_kind_of(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? fp_kind_of(job.fp_formats[1]) : -1;
     BlockSel bs{};
     bs.choice = choice;
     bs.block_sse = block_sse;
@@ -1267,22 +1297,12 @@ int launch_select_blocks(const ScoreJob &job, uint8_t *choice, float *block_sse,
     }
     fin.nc += 1;
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
-#define MOFQ_BLK(DT_, NI_, K0_, K1_)                                                                              \
-    if (x.dtype == DT_ && job.cs.n_int == NI_ && k0 == K0_ && k1 == K1_) {                                        \
-        kq_select_blocks<DT_, NI_, K0_, K1_><<<grid, 256, 0, st>>>(xp, x.rows, (int)x.cols, x.ld, width, team, rq, bs, job.hdr, \
-                                                                    job.partials, fin);                          \
-        MOFQ_CUDA_OK(cudaGetLastError());                                                                         \
-        return MOFQ_OK;                                                                                           \
-    }
-#define MOFQ_BLK_DT(DT_)                                                                                          \
-    MOFQ_BLK(DT_, 1, -1, -1) MOFQ_BLK(DT_, 0, 0, -1) MOFQ_BLK(DT_, 1, 0, -1) MOFQ_BLK(DT_, 0, 0, 0) MOFQ_BLK(DT_, 1, 0, 0) \
-    MOFQ_BLK(DT_, 0, 1, -1) MOFQ_BLK(DT_, 1, 1, -1) MOFQ_BLK(DT_, 0, 2, -1) MOFQ_BLK(DT_, 1, 2, -1)               \
-    MOFQ_BLK(DT_, 0, 1, 2) MOFQ_BLK(DT_, 1, 1, 2) MOFQ_BLK(DT_, 0, 2, 1) MOFQ_BLK(DT_, 1, 2, 1)
-    MOFQ_BLK_DT(0)
-    MOFQ_BLK_DT(1)
-#undef MOFQ_BLK_DT
-#undef MOFQ_BLK
-    return MOFQ_ERR_UNSUPPORTED;
+    return dispatch_kinds(x.dtype, job.cs.n_int, k0, k1, [&](auto DT, auto NI, auto K0, auto K1) {
+        kq_select_blocks<DT(), NI(), K0(), K1()><<<grid, 256, 0, st>>>(xp, x.rows, (int)x.cols, x.ld, width, team, rq, bs, job.hdr,
+                                                                       job.partials, fin);
+        MOFQ_CUDA_OK(cudaGetLastError());
+        return MOFQ_OK;
+    });
 }
 
 int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st)
@@ -1331,16 +1351,11 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
     p.stage_bytes = (best_r * row_bytes + 1023) & ~1023;
     p.stages = 3 * p.stage_bytes + 2048 <= 113 * 1024 ? 3 : 2;   // keep two blocks per SM
     p.grp_first = (job.gran == MOFQ_PER_GROUP) ? 1 : 0;
-    if (job.cs.n_int) p.rq.q[0] = job.cs.int_q;
-    for (int f = 0; f < job.cs.n_fp; ++f) p.rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
-    for (int j = 0; j < 3; ++j) p.rq.rq[j] = p.rq.q[j] > 0.0f ? 1.0f / p.rq.q[j] : 0.0f;
+    p.rq = job_rowq(job);
     p.n_tiles = (x.rows + best_r - 1) / best_r;
     const size_t smem = (size_t)p.stages * p.stage_bytes + 1024;
     const int threads = best_t + 32;
-    auto kind = [](int format) {
-        return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
-    };
-    const int k0 = job.cs.n_fp > 0 ? kind(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? kind(job.fp_formats[1]) : -1;
+    const int k0 = job.cs.n_fp > 0 ? fp_kind_of(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? fp_kind_of(job.fp_formats[1]) : -1;
     auto launch = [&](auto kernel) {
         if (int rc = set_smem(kernel, smem)) return rc;
         const int occ = std::max(1, blocks_per_sm((const void *)kernel, threads, smem));
@@ -1351,20 +1366,10 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
         MOFQ_CUDA_OK(cudaGetLastError());
         return MOFQ_OK;
     };
-#define MOFQ_RS(DT_, NI_, K0_, K1_)                                                                     \
-    if (x.dtype == DT_ && job.cs.n_int == NI_ && k0 == K0_ && k1 == K1_) {                              \
-        if (has_grp) return launch(kq_score_rows_stream<DT_, NI_, K0_, K1_, true>);                     \
-        return launch(kq_score_rows_stream<DT_, NI_, K0_, K1_, false>);                                 \
-    }
-#define MOFQ_RS_DT(DT_)                                                                                          \
-    MOFQ_RS(DT_, 1, -1, -1) MOFQ_RS(DT_, 0, 0, -1) MOFQ_RS(DT_, 1, 0, -1) MOFQ_RS(DT_, 0, 0, 0) MOFQ_RS(DT_, 1, 0, 0) \
-    MOFQ_RS(DT_, 0, 1, -1) MOFQ_RS(DT_, 1, 1, -1) MOFQ_RS(DT_, 0, 2, -1) MOFQ_RS(DT_, 1, 2, -1)                         \
-    MOFQ_RS(DT_, 0, 1, 2) MOFQ_RS(DT_, 1, 1, 2) MOFQ_RS(DT_, 0, 2, 1) MOFQ_RS(DT_, 1, 2, 1)
-    MOFQ_RS_DT(0)
-    MOFQ_RS_DT(1)
-#undef MOFQ_RS_DT
-#undef MOFQ_RS
-    return MOFQ_ERR_UNSUPPORTED;
+    return dispatch_kinds(x.dtype, job.cs.n_int, k0, k1, [&](auto DT, auto NI, auto K0, auto K1) {
+        if (has_grp) return launch(kq_score_rows_stream<DT(), NI(), K0(), K1(), true>);
+        return launch(kq_score_rows_stream<DT(), NI(), K0(), K1(), false>);
+    });
 }
 
 }  // namespace
@@ -1392,28 +1397,13 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
         else
             kq_absmax<1><<<grid, 256, 0, st>>>(xp, rows, (int)cpr, x.ld, job.hdr);
         MOFQ_CUDA_OK(cudaGetLastError());
-        RowQ rq{};
-        if (job.cs.n_int) rq.q[0] = job.cs.int_q;
-        for (int f = 0; f < job.cs.n_fp; ++f) rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
-        auto kind = [](int format) {
-            return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
-        };
-        const int k0 = job.cs.n_fp > 0 ? kind(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? kind(job.fp_formats[1]) : -1;
-#define MOFQ_UNI(DT_, NI_, K0_, K1_)                                                                                      \
-    if (x.dtype == DT_ && job.cs.n_int == NI_ && k0 == K0_ && k1 == K1_) {                                                \
-        kq_score_uniform<DT_, NI_, K0_, K1_><<<grid, 256, 0, st>>>(xp, rows, (int)cpr, x.ld, rq, job.hdr, job.partials, job.fin); \
-        MOFQ_CUDA_OK(cudaGetLastError());                                                                                 \
-        return MOFQ_OK;                                                                                                   \
-    }
-#define MOFQ_UNI_DT(DT_)                                                                                                  \
-    MOFQ_UNI(DT_, 1, -1, -1) MOFQ_UNI(DT_, 0, 0, -1) MOFQ_UNI(DT_, 1, 0, -1) MOFQ_UNI(DT_, 0, 0, 0) MOFQ_UNI(DT_, 1, 0, 0) \
-    MOFQ_UNI(DT_, 0, 1, -1) MOFQ_UNI(DT_, 1, 1, -1) MOFQ_UNI(DT_, 0, 2, -1) MOFQ_UNI(DT_, 1, 2, -1)                     \
-    MOFQ_UNI(DT_, 0, 1, 2) MOFQ_UNI(DT_, 1, 1, 2) MOFQ_UNI(DT_, 0, 2, 1) MOFQ_UNI(DT_, 1, 2, 1)
-        MOFQ_UNI_DT(0)
-        MOFQ_UNI_DT(1)
-#undef MOFQ_UNI_DT
-#undef MOFQ_UNI
-        return MOFQ_ERR_UNSUPPORTED;
+        const RowQ rq = job_rowq(job);
+        const int k0 = job.cs.n_fp > 0 ? fp_kind_of(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? fp_kind_of(job.fp_formats[1]) : -1;
+        return dispatch_kinds(x.dtype, job.cs.n_int, k0, k1, [&](auto DT, auto NI, auto K0, auto K1) {
+            kq_score_uniform<DT(), NI(), K0(), K1()><<<grid, 256, 0, st>>>(xp, rows, (int)cpr, x.ld, rq, job.hdr, job.partials, job.fin);
+            MOFQ_CUDA_OK(cudaGetLastError());
+            return MOFQ_OK;
+        });
     }
 
     // group scales only (dense or strided): the register-resident team kernel, without a format map
@@ -1428,13 +1418,8 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
     const size_t smem = (size_t)x.cols * 2 + (((size_t)chunks * 2 + 15) & ~(size_t)15) + (size_t)gpr * 8 * 3 + 16;
     if (smem > 200 * 1024) return MOFQ_ERR_UNSUPPORTED;
     const int grp_first = (job.gran == MOFQ_PER_GROUP) ? 1 : 0;
-    RowQ rq{};
-    if (job.cs.n_int) rq.q[0] = job.cs.int_q;
-    for (int f = 0; f < job.cs.n_fp; ++f) rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
-    auto kind = [](int format) {
-        return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
-    };
-    const int k0 = job.cs.n_fp > 0 ? kind(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? kind(job.fp_formats[1]) : -1;
+    const RowQ rq = job_rowq(job);
+    const int k0 = job.cs.n_fp > 0 ? fp_kind_of(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? fp_kind_of(job.fp_formats[1]) : -1;
     auto launch = [&](auto kernel) {
         if (int rc = set_smem(kernel, smem)) return rc;
         const int occ = std::max(1, blocks_per_sm((const void *)kernel, kRowThreads, smem));
@@ -1444,20 +1429,10 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
         MOFQ_CUDA_OK(cudaGetLastError());
         return MOFQ_OK;
     };
-#define MOFQ_ROWS(DT_, NI_, K0_, K1_)                                                                   \
-    if (x.dtype == DT_ && job.cs.n_int == NI_ && k0 == K0_ && k1 == K1_) {                              \
-        if (has_ch && has_grp) return launch(kq_score_rows<DT_, NI_, K0_, K1_, true, true>);            \
-        return launch(kq_score_rows<DT_, NI_, K0_, K1_, true, false>);                                  \
-    }
-#define MOFQ_ROWS_DT(DT_)                                                                                        \
-    MOFQ_ROWS(DT_, 1, -1, -1) MOFQ_ROWS(DT_, 0, 0, -1) MOFQ_ROWS(DT_, 1, 0, -1) MOFQ_ROWS(DT_, 0, 0, 0) MOFQ_ROWS(DT_, 1, 0, 0) \
-    MOFQ_ROWS(DT_, 0, 1, -1) MOFQ_ROWS(DT_, 1, 1, -1) MOFQ_ROWS(DT_, 0, 2, -1) MOFQ_ROWS(DT_, 1, 2, -1)                         \
-    MOFQ_ROWS(DT_, 0, 1, 2) MOFQ_ROWS(DT_, 1, 1, 2) MOFQ_ROWS(DT_, 0, 2, 1) MOFQ_ROWS(DT_, 1, 2, 1)
-    MOFQ_ROWS_DT(0)
-    MOFQ_ROWS_DT(1)
-#undef MOFQ_ROWS_DT
-#undef MOFQ_ROWS
-    return MOFQ_ERR_UNSUPPORTED;
+    return dispatch_kinds(x.dtype, job.cs.n_int, k0, k1, [&](auto DT, auto NI, auto K0, auto K1) {
+        if (has_ch && has_grp) return launch(kq_score_rows<DT(), NI(), K0(), K1(), true, true>);
+        return launch(kq_score_rows<DT(), NI(), K0(), K1(), true, false>);
+    });
 }
 
 // Per-tensor scale from the abs-max already stored in hdr->absmax_bits (launch_absmax); codes of n formats from one read.
