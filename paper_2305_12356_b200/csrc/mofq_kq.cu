@@ -448,6 +448,10 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
     }
     if (tid < 8 * kRsMaxRows) (&rowmax[0][0])[tid] = 0;
     __syncthreads();
+    // Programmatic dependent launch: the next launch on the stream (the next layer's scoring) may start as soon as
+    // every block of this one is running, so its blocks fill the SMs this launch's tail leaves idle.  Its reads are
+    // of its own input only; it waits for this launch to complete (below) before touching the shared workspace.
+    asm volatile("griddepcontrol.launch_dependents;");
     const long long t_begin = (long long)blockIdx.x * p.tiles_per_cta;
     const long long t_end = min(t_begin + p.tiles_per_cta, p.n_tiles);
     const int n_it = t_end > t_begin ? (int)(t_end - t_begin) : 0;
@@ -486,10 +490,25 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
         }
     } else {
         // ---------------- consumers ----------------
+        // a thread's segments sit at the same place in every tile: row within the tile and byte offset, once
+        int seg_row[2];
+        uint32_t seg_off[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int g = tid + k * p.consumers;
+            seg_row[k] = g / p.segs_per_row;
+            seg_off[k] = (uint32_t)seg_row[k] * row_bytes + (uint32_t)(g - seg_row[k] * p.segs_per_row) * 256u + (uint32_t)((tid & 15) << 4);
+        }
+        int s1 = 0;            // stage and phase of the tile pass 1 takes next
+        uint32_t ph1 = 0;
         // pass 1 of tile `it`: abs-max of this thread's segments, folded into the tile's per-row maxima
         auto pass1 = [&](int it, RsSeg &sg) {
-            const int s = it % p.stages;
-            const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+            const int s = s1;
+            const uint32_t ph = ph1;
+            if (++s1 == p.stages) {
+                s1 = 0;
+                ph1 ^= 1u;
+            }
             const bool ok = mbar_wait(&full_bar[s], ph, &err);
             const long long r0 = (t_begin + it) * p.rows_per_tile;
             const int nr = (int)min((long long)p.rows_per_tile, p.rows - r0);
@@ -503,8 +522,8 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
                 sg.segmax[k] = 0;
                 sg.row[k] = 0;
                 if (g < nseg) {
-                    sg.row[k] = g / p.segs_per_row;
-                    sg.a0[k] = tile + (uint32_t)sg.row[k] * row_bytes + (uint32_t)(g - sg.row[k] * p.segs_per_row) * 256u + (uint32_t)((tid & 15) << 4);
+                    sg.row[k] = seg_row[k];
+                    sg.a0[k] = tile + seg_off[k];
                     uint32_t m = 0;
 #pragma unroll
                     for (int j = 0; j < 16; ++j) m = kqmath::absmax_chunk<DT>(lds128(sg.a0[k] ^ (uint32_t)(j << 4)), m);
@@ -517,6 +536,7 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
         };
         RsSeg cur, nxt;
         if (n_it > 0) pass1(0, cur);
+        int s2 = 0;            // stage pass 2 releases next
         for (int it = 0; it < n_it; ++it) {
             if (it + 1 < n_it) pass1(it + 1, nxt);
             const bool ok = mbar_wait(&row_bar[it & 1], (uint32_t)(it >> 1) & 1u, &err);   // every warp has finished pass 1 of this tile
@@ -568,10 +588,14 @@ kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[it % p.stages]);
+            if (lane == 0) mbar_arrive(&empty_bar[s2]);
+            if (++s2 == p.stages) s2 = 0;
             cur = nxt;
         }
     }
+    // the previous launch on the stream has finished with the header and the partial sums once this returns
+    // (a no-op when this launch was not started early)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     block_finish<NA>(dacc, status, hdr, partials, fin, red);
 }
 
@@ -1326,18 +1350,37 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
     const mofq_tensor &x = job.x;
     const int spr = (int)(x.cols / 128);
     const int row_bytes = (int)x.cols * 2;
-    // tile shape: as many whole rows as fit in 36 KB (three stages of that leave room for two blocks per SM), at
-    // most two 128-element segments per consumer thread, consumers a multiple of 32
-    int best_r = 1;
-    while (best_r < kRsMaxRows && (long long)(best_r + 1) <= x.rows && (best_r + 1) * row_bytes <= 36864) ++best_r;
-    int best_t = 0;
-    for (; best_r >= 1 && !best_t; --best_r) {
-        const int nseg = best_r * spr;
-        for (int rounds = 1; rounds <= 2 && !best_t; ++rounds) {
+    // tile shape: as many whole rows as fit in 36 KB, at most two 128-element segments per consumer thread,
+    // consumers a multiple of 32
+    auto consumers_for = [&](int r, int max_rounds, int *rounds_out) {
+        const int nseg = r * spr;
+        for (int rounds = 1; rounds <= max_rounds; ++rounds) {
             const int t = 32 * ((nseg + 32 * rounds - 1) / (32 * rounds));
-            if (t <= kRsMaxConsumers) best_t = t;
+            if (t <= kRsMaxConsumers) {
+                *rounds_out = rounds;
+                return t;
+            }
         }
-        if (best_t) break;
+        return 0;
+    };
+    int best_r = 1, best_t = 0, best_rounds = 1;
+    while (best_r < kRsMaxRows && (long long)(best_r + 1) <= x.rows && (best_r + 1) * row_bytes <= 36864) ++best_r;
+    for (; best_r >= 1; --best_r)
+        if ((best_t = consumers_for(best_r, 2, &best_rounds)) != 0) break;
+    if (best_t && has_grp) {
+        // With two scale sets per element the lanes of a partly filled last warp cost the most: take a taller tile
+        // (two stages of up to 52 KB still leave two blocks per SM) when it fills the warps clearly better
+        // (6656-element rows: 104 of 128 lanes with two rows, 208 of 224 with four).
+        double util = (double)(best_r * spr) / (double)(best_t * best_rounds);
+        for (int r = best_r + 1; r <= kRsMaxRows && r <= x.rows && r * row_bytes <= 53248; ++r) {
+            int rounds = 1;
+            const int t = consumers_for(r, 1, &rounds);
+            if (t && (double)(r * spr) / t > util + 0.1) {
+                util = (double)(r * spr) / t;
+                best_r = r;
+                best_t = t;
+            }
+        }
     }
     if (!best_t) return MOFQ_ERR_UNSUPPORTED;
     RsParams p{};
@@ -1350,6 +1393,10 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
     p.consumers = best_t;
     p.stage_bytes = (best_r * row_bytes + 1023) & ~1023;
     p.stages = 3 * p.stage_bytes + 2048 <= 113 * 1024 ? 3 : 2;   // keep two blocks per SM
+    // With two scale sets per element more resident warps hide more than a third stage does: two stages when that
+    // fits four blocks per SM (measured, 3 -> 2 stages: 6656-element rows 138.7 -> 129.7 us on 17920 rows,
+    // 11008-element rows 65.4 -> 55.0 us on 4096 rows).  The taller tiles above only fit with two anyway.
+    if (has_grp && 2 * p.stage_bytes + 2048 <= 56 * 1024) p.stages = 2;
     p.grp_first = (job.gran == MOFQ_PER_GROUP) ? 1 : 0;
     p.rq = job_rowq(job);
     p.n_tiles = (x.rows + best_r - 1) / best_r;
@@ -1362,8 +1409,18 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
         long long grid = std::min<long long>(p.n_tiles, std::min<long long>((long long)sm_count() * occ, kMaxSlots));
         p.tiles_per_cta = (p.n_tiles + grid - 1) / grid;
         grid = (p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
-        kernel<<<(int)grid, threads, smem, st>>>(p, job.hdr, job.partials, job.fin);
-        MOFQ_CUDA_OK(cudaGetLastError());
+        // allowed to start before the previous kernel on the stream has drained (see the kernel's griddepcontrol pair)
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3((unsigned)grid);
+        lc.blockDim = dim3((unsigned)threads);
+        lc.dynamicSmemBytes = smem;
+        lc.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at;
+        lc.numAttrs = 1;
+        MOFQ_CUDA_OK(cudaLaunchKernelEx(&lc, kernel, p, job.hdr, job.partials, job.fin));
         return MOFQ_OK;
     };
     return dispatch_kinds(x.dtype, job.cs.n_int, k0, k1, [&](auto DT, auto NI, auto K0, auto K1) {

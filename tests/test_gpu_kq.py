@@ -372,6 +372,33 @@ def test_streamed_rows_shapes(orc, dev, rows, cols, ld):
     assert rel_err(got2.cpu().numpy().reshape(-1), want2).max() < MSE_RTOL
 
 
+def test_streamed_rows_back_to_back_launches_share_one_workspace(orc, dev):
+    """The streamed-row kernel lets the next launch on the stream start before it has drained; the header and the
+    partial sums they share are only touched after the earlier launch has completed.  Many short launches in a row
+    (different tensors, one workspace, no host synchronisation) must give what each gives when launched alone."""
+    names = ["INT4", "FP4_E2M1"]
+    shapes = [(300, 6656), (17, 4096), (640, 1024), (96, 17920), (1, 128), (410, 6656)]
+    xs = [_weights(dev, r, c, seed=43, layer=i) for i, (r, c) in enumerate(shapes)]
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device=dev)
+    alone = []
+    for x in xs:
+        got, st = mofq.tensor_error(x, names, "channel", gran2="group", group=128, workspace=ws)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        alone.append(got.cpu().numpy().copy())
+    want0 = np.concatenate([_oracle_mse(orc, host(xs[0]), names, "channel", 0), _oracle_mse(orc, host(xs[0]), names, "group", 128)])
+    assert rel_err(alone[0].reshape(-1), want0).max() < MSE_RTOL
+    for _ in range(3):
+        outs = []
+        for rep in range(4):
+            for x in xs:
+                outs.append(mofq.tensor_error(x, names, "channel", gran2="group", group=128, workspace=ws)[0])
+        torch.cuda.synchronize()
+        assert int(ws[:4].view(torch.int32).item()) == 0
+        for k, o in enumerate(outs):
+            np.testing.assert_array_equal(o.cpu().numpy().view(np.uint32), alone[k % len(xs)].view(np.uint32))
+
+
 @pytest.mark.parametrize("name", FMT4 + FMT8)
 def test_fast_scale_pair_is_correctly_rounded_for_every_binary16_magnitude(orc, dev, name):
     from paper_2305_12356_b200.binding import diag_scale_pair
