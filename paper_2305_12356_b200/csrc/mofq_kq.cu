@@ -1409,7 +1409,8 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
         long long grid = std::min<long long>(p.n_tiles, std::min<long long>((long long)sm_count() * occ, kMaxSlots));
         p.tiles_per_cta = (p.n_tiles + grid - 1) / grid;
         grid = (p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
-        // allowed to start before the previous kernel on the stream has drained (see the kernel's griddepcontrol pair)
+        // After another scoring launch of the same call this one may start before that one has drained (see the
+        // kernel's griddepcontrol pair); after anything else on the stream it starts in stream order as usual.
         cudaLaunchConfig_t lc{};
         lc.gridDim = dim3((unsigned)grid);
         lc.blockDim = dim3((unsigned)threads);
@@ -1419,7 +1420,7 @@ int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
         at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         at[0].val.programmaticStreamSerializationAllowed = 1;
         lc.attrs = at;
-        lc.numAttrs = 1;
+        lc.numAttrs = job.overlap_prev ? 1 : 0;
         MOFQ_CUDA_OK(cudaLaunchKernelEx(&lc, kernel, p, job.hdr, job.partials, job.fin));
         return MOFQ_OK;
     };

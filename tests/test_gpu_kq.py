@@ -372,31 +372,37 @@ def test_streamed_rows_shapes(orc, dev, rows, cols, ld):
     assert rel_err(got2.cpu().numpy().reshape(-1), want2).max() < MSE_RTOL
 
 
-def test_streamed_rows_back_to_back_launches_share_one_workspace(orc, dev):
-    """The streamed-row kernel lets the next launch on the stream start before it has drained; the header and the
-    partial sums they share are only touched after the earlier launch has completed.  Many short launches in a row
-    (different tensors, one workspace, no host synchronisation) must give what each gives when launched alone."""
+def test_streamed_rows_layers_of_one_call_overlap_safely(orc, dev):
+    """Within one selection call the streamed-row kernel lets the next layer's launch start before the current one has
+    drained; the header and the partial sums they share are only touched after the earlier launch has completed.
+    Many short layers in one call, and calls back to back without host synchronisation, must give for every layer
+    exactly what that layer gives when scored alone."""
     names = ["INT4", "FP4_E2M1"]
-    shapes = [(300, 6656), (17, 4096), (640, 1024), (96, 17920), (1, 128), (410, 6656)]
-    xs = [_weights(dev, r, c, seed=43, layer=i) for i, (r, c) in enumerate(shapes)]
+    shapes = [(300, 6656), (17, 4096), (640, 1024), (96, 17920), (1, 128), (410, 6656)] * 4
+    xs = [_weights(dev, r, c, seed=43, layer=i % 6) for i, (r, c) in enumerate(shapes)]
     ws = torch.zeros(1 << 20, dtype=torch.uint8, device=dev)
     alone = []
-    for x in xs:
+    for x in xs[:6]:
         got, st = mofq.tensor_error(x, names, "channel", gran2="group", group=128, workspace=ws)
         torch.cuda.synchronize()
         assert int(st.item()) == 0
         alone.append(got.cpu().numpy().copy())
     want0 = np.concatenate([_oracle_mse(orc, host(xs[0]), names, "channel", 0), _oracle_mse(orc, host(xs[0]), names, "group", 128)])
     assert rel_err(alone[0].reshape(-1), want0).max() < MSE_RTOL
-    for _ in range(3):
-        outs = []
-        for rep in range(4):
-            for x in xs:
-                outs.append(mofq.tensor_error(x, names, "channel", gran2="group", group=128, workspace=ws)[0])
-        torch.cuda.synchronize()
-        assert int(ws[:4].view(torch.int32).item()) == 0
-        for k, o in enumerate(outs):
-            np.testing.assert_array_equal(o.cpu().numpy().view(np.uint32), alone[k % len(xs)].view(np.uint32))
+    cfg = mofq.make_config(4, names, w_gran="channel", w_group=128, w_gran2="group")
+    prepared = mofq.prepare_layers(xs)
+    wsel = torch.zeros(mofq.workspace_bytes(prepared, cfg), dtype=torch.uint8, device=dev)
+    raw = [torch.empty(2 * len(xs) * B.RESULT_BYTES, dtype=torch.uint8, device=dev) for _ in range(3)]
+    for out in raw:                                         # three calls in a row, nothing synchronises in between
+        mofq.select_formats(prepared, cfg, workspace=wsel, results=out, parse=False)
+    torch.cuda.synchronize()
+    for out in raw:
+        recs = B._parse_results(bytes(out.cpu().numpy()), 2 * len(xs), len(names))
+        for li in range(len(xs)):
+            for s_ in range(2):
+                r = recs[2 * li + s_]
+                assert r["status"] == 0
+                np.testing.assert_array_equal(np.asarray(r["errors"], np.float32).view(np.uint32), alone[li % 6][s_].view(np.uint32))
 
 
 @pytest.mark.parametrize("name", FMT4 + FMT8)
