@@ -404,7 +404,7 @@ int mofq_emit_selected(const mofq_layer *layers, int n_layers, const mofq_config
         sel.res = results + (size_t)i * n_sets;
         sel.tag_out = formats_out ? formats_out + i : nullptr;
         if (int rc = launch_emit(layers[i].W, sel.cand[0], cfg->w_gran, cfg->w_group, nullptr, out[i].codes, out[i].scales, nullptr,
-                                 nullptr, MOFQ_F16, static_cast<WsHeader *>(workspace), st, -1, &sel))
+                                 nullptr, MOFQ_F16, static_cast<WsHeader *>(workspace), st, -1, &sel, i > 0))
             return rc;
     }
     return MOFQ_OK;

@@ -111,7 +111,8 @@ int launch_select_blocks(const ScoreJob &job, uint8_t *choice, float *block_sse,
 int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in,
                 void *codes_out, float *scales_out, void *dequant_out, void *values_out, int values_dtype,
                 WsHeader *hdr, cudaStream_t st, int format_id = -1 /* mofq_format of f: enables the fused code kernel */,
-                const EmitSel *sel = nullptr /* format chosen on the device; f then only fixes the code width */);
+                const EmitSel *sel = nullptr /* format chosen on the device; f then only fixes the code width */,
+                bool overlap_prev = false /* the previous launch on st is the previous layer's emission of the same call */);
 int launch_emit_codes_uniform(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
                               WsHeader *hdr, cudaStream_t st);
 int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,

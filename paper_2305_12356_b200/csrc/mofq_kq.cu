@@ -792,6 +792,10 @@ kq_emit(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, 
         uint16_t *values_out, int values_dtype, WsHeader *hdr, const EmitSel sel)
 {
     __shared__ uint32_t mred[34];
+    // When the host launched this kernel as the next layer of one emission call, the launch after it may start as
+    // soon as every block of this one is running: the layers read and write disjoint buffers.  The wait at the end
+    // keeps the launches completing in stream order.
+    asm volatile("griddepcontrol.launch_dependents;");
     if (sel.res) {  // the winner of the selection record decides the grid
         const int c = min(max(sel.res->chosen, 0), MOFQ_MAX_CAND - 1);
         f = sel.cand[c];
@@ -1062,6 +1066,10 @@ __global__ void __launch_bounds__(256)
 kq_emit_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, FmtDesc f, int width, int uniform,
                unsigned char *codes_out, float *scales_out, WsHeader *hdr, const EmitSel sel)
 {
+    // When the host launched this kernel as the next layer of one emission call, the launch after it may start as
+    // soon as every block of this one is running: the layers read and write disjoint buffers.  The wait at the end
+    // keeps the launches completing in stream order.
+    asm volatile("griddepcontrol.launch_dependents;");
     if (sel.res) {  // the winner of the selection record decides the grid
         const int c = min(max(sel.res->chosen, 0), MOFQ_MAX_CAND - 1);
         f = sel.cand[c];
@@ -1076,6 +1084,7 @@ kq_emit_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long lo
     case CLS_E4M3: emit_blocks<DT, CLS_E4M3>(x, rows, cols, ld, f.Q, width, uniform != 0, codes_out, scales_out, hdr, status); break;
     default: emit_blocks<DT, CLS_E5M2>(x, rows, cols, ld, f.Q, width, uniform != 0, codes_out, scales_out, hdr, status); break;
     }
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // a no-op unless this launch was started early
     if (status) atomicOr(&hdr->status, status);
 }
 
@@ -1554,7 +1563,7 @@ int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void
 
 int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in, void *codes_out,
                 float *scales_out, void *dequant_out, void *values_out, int values_dtype, WsHeader *hdr, cudaStream_t st,
-                int format_id, const EmitSel *sel)
+                int format_id, const EmitSel *sel, bool overlap_prev)
 {
     EmitSel es{};
     if (sel) {
@@ -1588,13 +1597,23 @@ int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, con
         const long long n_blocks = x.rows * (x.cols / width);
         const long long warps = (n_blocks + (32 / team) - 1) / (32 / team);
         const int g = (int)std::min<long long>((warps + 7) / 8, (long long)nsm * 8);
+        // group scales, after the previous layer's launch of the same emission call: may start while that one drains
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3((unsigned)g);
+        lc.blockDim = dim3(256);
+        lc.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at;
+        lc.numAttrs = (overlap_prev && gran == MOFQ_PER_GROUP) ? 1 : 0;
+        const int uniform = gran == MOFQ_PER_TENSOR ? 1 : 0;
         if (x.dtype == MOFQ_F16)
-            kq_emit_blocks<0><<<g, 256, 0, st>>>(xp, x.rows, (int)x.cols, x.ld, f, width, gran == MOFQ_PER_TENSOR,
-                                                 (unsigned char *)codes_out, scales_out, hdr, es);
+            MOFQ_CUDA_OK(cudaLaunchKernelEx(&lc, kq_emit_blocks<0>, xp, (long long)x.rows, (int)x.cols, (long long)x.ld, f, width, uniform,
+                                            (unsigned char *)codes_out, scales_out, hdr, es));
         else
-            kq_emit_blocks<1><<<g, 256, 0, st>>>(xp, x.rows, (int)x.cols, x.ld, f, width, gran == MOFQ_PER_TENSOR,
-                                                 (unsigned char *)codes_out, scales_out, hdr, es);
-        MOFQ_CUDA_OK(cudaGetLastError());
+            MOFQ_CUDA_OK(cudaLaunchKernelEx(&lc, kq_emit_blocks<1>, xp, (long long)x.rows, (int)x.cols, (long long)x.ld, f, width, uniform,
+                                            (unsigned char *)codes_out, scales_out, hdr, es));
         return MOFQ_OK;
     }
     const int grid = (int)std::min<long long>(x.rows, (long long)nsm * 8);
