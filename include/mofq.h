@@ -195,6 +195,10 @@ int mofq_layer_output_error(const mofq_layer *L, const mofq_config *cfg, float *
  *   layers       host array of n_layers descriptors (device tensors)
  *   results_out  device array of n_layers records (2*n_layers when cfg->w_gran2 is given)
  *   workspace    at least mofq_workspace_bytes(layers, n_layers, cfg)
+ * The layers' kernels of one call may overlap on the device (a layer's launch can start while the previous
+ * layer's drains); seen from the stream the call is one unit: it starts after everything enqueued before
+ * it and everything enqueued after it sees all its records.  The output buffers of the layers
+ * (results_out here, codes / scales in mofq_emit_selected) must therefore not alias each other.
  */
 int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_config *cfg,
                         mofq_result *results_out, void *workspace, size_t workspace_bytes, void *stream);
