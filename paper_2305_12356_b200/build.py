@@ -15,7 +15,7 @@ BUILD_DIR = os.path.join(_HERE, "_build")
 LIB = os.path.join(_HERE, "libmofq.so")
 SYNTH_LIB = os.path.join(_HERE, "libmofq_synth.so")
 
-LIB_SOURCES = ["mofq_kq.cu", "mofq_kq_mt.cu", "mofq_layer.cu", "mofq_api.cu", "mofq_noalloc.cu", "mofq_diag.cu"]
+LIB_SOURCES = ["mofq_kq.cu", "mofq_kq_mt.cu", "mofq_kq_rows.cu", "mofq_layer.cu", "mofq_api.cu", "mofq_noalloc.cu", "mofq_diag.cu"]
 SYNTH_SOURCES = ["mofq_synth.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

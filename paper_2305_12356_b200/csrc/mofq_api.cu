@@ -195,6 +195,7 @@ size_t mofq_workspace_bytes(const mofq_layer *layers, int n_layers, const mofq_c
     size_t need = align256(score_ws_bytes());
     if (cfg && cfg->metric == MOFQ_LAYER_OUTPUT_MSE && layers) need += layer_metric_ws_bytes(layers, n_layers, cfg);
     if (cfg && layers && n_layers > 0 && mt_applicable(layers, n_layers, cfg)) need += mt_ws_bytes(n_layers);
+    else if (cfg && layers && n_layers > 0 && rows_mt_applicable(layers, n_layers, cfg)) need += rows_mt_ws_bytes(n_layers);
     return need;
 }
 
@@ -368,6 +369,9 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
     if (mt_applicable(layers, n_layers, cfg))  // one persistent launch over the whole layer list
         return mt_run(layers, n_layers, cfg, cs, perm, nc, fp_formats, results_out,
                       static_cast<char *>(workspace) + align256(score_ws_bytes()), st);
+    if (rows_mt_applicable(layers, n_layers, cfg))  // per-channel scales: one persistent launch over whole-row tiles
+        return rows_mt_run(layers, n_layers, cfg, cs, perm, nc, fp_formats, results_out,
+                           static_cast<char *>(workspace) + align256(score_ws_bytes()), st);
     if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
     const int n_sets = cfg->w_gran2 != MOFQ_GRAN_NONE ? 2 : 1;
     for (int i = 0; i < n_layers; ++i) {  // Algorithm 1: for layer in model.layers_to_quant

@@ -29,6 +29,20 @@ struct CandSet {
     uint32_t fp_eminb[2], fp_kadd[2];
 };
 
+// abs-max targets of a candidate set's canonical slots and their rounded reciprocals (for the division-free scales)
+struct RowQ {
+    float q[3];   // abs-max target per canonical slot
+    float rq[3];  // RN32(1 / q)
+};
+inline RowQ candset_rowq(const CandSet &cs)
+{
+    RowQ rq{};
+    if (cs.n_int) rq.q[0] = cs.int_q;
+    for (int f = 0; f < cs.n_fp; ++f) rq.q[cs.n_int + f] = cs.fp_q[f];
+    for (int j = 0; j < 3; ++j) rq.rq[j] = rq.q[j] > 0.0f ? 1.0f / rq.q[j] : 0.0f;
+    return rq;
+}
+
 constexpr int kMaxAcc = 8;        // accumulators per block: up to 2 granularities x 3 canonical slots (padded)
 constexpr int kMaxSlots = 2048;   // most thread blocks a scoring kernel is launched with
 
@@ -91,6 +105,14 @@ int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const
            const int *fp_formats, mofq_result *results /* nullable */, void *ws, cudaStream_t st,
            float *mse_out = nullptr /* [layer][candidate] */, int32_t *status_out = nullptr /* OR of the layers' status bits */);
 int sm_count();
+
+// streamed-rows path (mofq_kq_rows.cu): per-channel scales, alone or with group-128 scales from the same read
+bool rows_single_applicable(const ScoreJob &job);
+int rows_single_run(const ScoreJob &job, cudaStream_t st);
+bool rows_mt_applicable(const mofq_layer *layers, int n_layers, const mofq_config *cfg);
+size_t rows_mt_ws_bytes(int n_layers);
+int rows_mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
+                const int *fp_formats, mofq_result *results, void *ws, cudaStream_t st);
 
 // Format of an emit launch picked ON THE DEVICE from a selection record (Algorithm 1's last step without a host
 // round trip): the kernel quantises with cand[res->chosen] and stores that candidate's mofq_format in *tag_out.

@@ -14,12 +14,15 @@
 #include <cstring>
 #include <type_traits>
 
+#include "kq_finish.cuh"
 #include "kq_math.cuh"
 #include "kq_pipe.cuh"
 #include "mofq_internal.h"
 
 namespace mofq {
 namespace {
+
+using kqfin::write_outputs;
 
 constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds |t| < 2^22 to an integer (RNE)
 
@@ -111,43 +114,6 @@ __device__ __forceinline__ void block_sum(double *acc, double *red /* >= 32*NA +
     __syncthreads();
 }
 
-__device__ void write_outputs(const double *tot, const Finalize &fin, WsHeader *hdr)
-{
-    int status = 0;
-    if (fin.res) status = atomicExch(&hdr->status, 0);
-    for (int s = 0; s < fin.n_sets; ++s) {
-        double err[MOFQ_MAX_CAND];
-        for (int i = 0; i < fin.n_cand; ++i) {
-            err[i] = tot[s * fin.nc + fin.perm[i]] * fin.inv_n;
-            if (fin.mse_out) fin.mse_out[s * fin.n_cand + i] = (float)err[i];
-        }
-        if (fin.res) {
-            // Algorithm 1: min_error = inf; replace only on a strictly smaller error, caller's order
-            double best = INFINITY, second = INFINITY;
-            int chosen = -1;
-            for (int i = 0; i < fin.n_cand; ++i) {
-                if (err[i] < best) {
-                    second = best;
-                    best = err[i];
-                    chosen = i;
-                } else if (err[i] < second) {
-                    second = err[i];
-                }
-            }
-            mofq_result r;
-            r.chosen = chosen;
-            r.status = status;
-            for (int i = 0; i < MOFQ_MAX_CAND; ++i) {
-                r.error[i] = i < fin.n_cand ? (float)err[i] : 0.0f;
-                r.nsr[i] = 0.0f;
-            }
-            r.rel_margin = best > 0.0 ? (float)((second - best) / best) : INFINITY;
-            r.reserved = 0;
-            fin.res[s] = r;
-        }
-    }
-}
-
 // Every block deposits its partial sums; the block that arrives last adds them in slot order.
 template <int NA>
 __device__ void block_finish(double *acc, int status, WsHeader *hdr, double *partials, const Finalize &fin, double *red)
@@ -186,11 +152,6 @@ __device__ void block_finish(double *acc, int status, WsHeader *hdr, double *par
 // Arithmetic: packed f32x2 and hardware FP converts (kq_math.cuh).  Accumulator order: [first set][second
 // set]; `grp_first` says whether the group set comes first.
 constexpr int kRowThreads = 256;
-
-struct RowQ {
-    float q[3];   // abs-max target per canonical slot
-    float rq[3];  // RN32(1 / q), for the division-free scale computation
-};
 
 template <int DT, int NI, int K0, int K1, bool CH, bool GRP>
 __global__ void __launch_bounds__(kRowThreads)
@@ -1229,15 +1190,7 @@ int fp_kind_of(int format)
     return format == MOFQ_FP8_E4M3 ? (int)kqmath::FPK_E4M3 : format == MOFQ_FP8_E5M2 ? (int)kqmath::FPK_E5M2 : (int)kqmath::FPK_E2M1;
 }
 
-// abs-max targets (and their reciprocals) of a job's canonical slots
-RowQ job_rowq(const ScoreJob &job)
-{
-    RowQ rq{};
-    if (job.cs.n_int) rq.q[0] = job.cs.int_q;
-    for (int f = 0; f < job.cs.n_fp; ++f) rq.q[job.cs.n_int + f] = job.cs.fp_q[f];
-    for (int j = 0; j < 3; ++j) rq.rq[j] = rq.q[j] > 0.0f ? 1.0f / rq.q[j] : 0.0f;
-    return rq;
-}
+RowQ job_rowq(const ScoreJob &job) { return candset_rowq(job.cs); }
 
 int blocks_per_sm(const void *kernel, int threads, size_t smem)
 {
@@ -1478,8 +1431,7 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
 
     // row kernels: per-channel scales, alone or with group scales from the same read
     if (x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
-    if (has_ch && x.cols % 128 == 0 && x.cols * 2 <= kRsMaxTileBytes && (!has_grp || job.group == 128))
-        return launch_score_rows_stream(job, has_grp, st);
+    if (rows_single_applicable(job)) return rows_single_run(job, st);
     const int chunks = (int)(x.cols / 8);
     const int gpr = has_grp ? (int)(x.cols / job.group) : 0;
     const size_t smem = (size_t)x.cols * 2 + (((size_t)chunks * 2 + 15) & ~(size_t)15) + (size_t)gpr * 8 * 3 + 16;
