@@ -14,12 +14,29 @@
  *     (a Linear layer's weight, A_out = W * A_in, Section 3.2); activations are [tokens, in].
  *   - `data` must be 16-byte aligned, `cols` a multiple of 8 and `ld` a multiple of 8.
  *   - The caller owns every buffer, the workspace included; the library allocates nothing and
- *     keeps no state between calls.  All work is enqueued on `stream` (a cudaStream_t passed as
- *     void*; NULL = default stream) and the call returns without synchronising, unless stated.
- *   - Return value: 0 on success, a negative MOFQ_ERR_* for a synchronous argument error (nothing
- *     was enqueued).  Conditions found on the device (non-finite input, a reciprocal scale that
- *     overflows binary32) are reported as MOFQ_STATUS_* bits in a device status word.
+ *     keeps no state between calls.  The one exception is mofq_tensor_error_noalloc, which works
+ *     in a fixed scratch array inside the library (see there).  All work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL = default stream) and the call returns without
+ *     synchronising, unless stated.
+ *   - Return value: 0 on success, a negative MOFQ_ERR_* for a synchronous argument error.  After
+ *     a negative return the call's outputs are not produced.  Pointer, size, alignment, enum,
+ *     candidate and workspace errors are found before anything is enqueued; a combination that
+ *     only a kernel's launcher can refuse (MOFQ_ERR_UNSUPPORTED for a per-tensor scale together
+ *     with a second granularity, rows too long for shared memory, more than 2^31 chunks) may be
+ *     found after the clear of the workspace header has been enqueued, and in
+ *     mofq_select_formats / mofq_emit_selected after the layers before the refused one.
+ *     Conditions found on the device (non-finite input, a reciprocal scale that overflows
+ *     binary32) are reported as MOFQ_STATUS_* bits in a device status word.
  *   - Input values must be finite.
+ *   - Candidates: at most MOFQ_MAX_CAND entries per call, of which at most one INT format and two
+ *     distinct FP formats (three distinct formats); a list may repeat a format.
+ *   - What the arithmetic contract below binds: the code-writing calls (mofq_quantize_tensor,
+ *     mofq_emit_selected) follow it operation by operation, so codes, scales and dequantised
+ *     values are determined bit for bit.  The scoring calls report errors that agree with the
+ *     contract's to within 1e-5 relative: they may fuse the multiply into the INT rounding and
+ *     form the FP candidates' differences in units of the scale, which can move a value only where
+ *     x * inv lies within one binary32 ulp of a rounding tie (where both neighbours have the same
+ *     error).
  *
  * Arithmetic contract (what "quantise" means here; the paper states round-to-nearest linear
  * quantisation with abs-max scales and leaves the rest open):
@@ -119,8 +136,7 @@ typedef struct {
 
 /*
  * mofq_quantize_tensor - round-to-nearest linear quantisation of one tensor to one format
- * (Section 1 "naive linear quantization with round-to-nearest", Algorithm 1 `quantize_layer`;
- * granularities Section 3.2).
+ * (the plain RTN quantiser of Section 1, Algorithm 1 `quantize_layer`; granularities Section 3.2).
  *   x           tensor to quantise
  *   scales_in   NULL: abs-max scales are derived.  Else device array of n_scales floats
  *               (calibration scales, Section 3.2 dynamic tensor analysis); values saturate.
@@ -137,9 +153,9 @@ int mofq_quantize_tensor(const mofq_tensor *x, int format, int gran, int group, 
                          void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * mofq_tensor_error - tensor MSE of n candidate formats of one bit-width from ONE read of x
- * (Section 3.2 static tensor analysis: "mean squared error between quantized and original
- * tensors"; Algorithm 1 `compute_error` with the tensor metric).
+ * mofq_tensor_error - tensor MSE (quantised against original tensor) of n candidate formats of one
+ * bit-width from ONE read of x (Section 3.2, static tensor analysis; Algorithm 1 `compute_error`
+ * with the tensor metric).
  *   formats     host array of n mofq_format values of equal bit-width
  *   gran2       MOFQ_GRAN_NONE or a second granularity scored from the same read
  *   mse_out     device, n floats (2n when gran2 is given: [gran][candidate])
@@ -174,7 +190,8 @@ int mofq_absmax_update(const mofq_tensor *x, float *absmax_inout, void *stream);
  * mofq_tensor_error_scaled - tensor MSE of n candidates under CALLER-SUPPLIED per-tensor scales, e.g. calibration scales
  * applied to an unseen activation batch (Section 3.2, dynamic tensor analysis).  scales_in: device, n floats, one scale
  * per candidate in the caller's order (typically calibration abs-max / format maximum); inv = RN32(1/scale); values
- * beyond the grid saturate.  mse_out: device, n floats.  workspace as for mofq_tensor_error.
+ * beyond the grid saturate.  Every candidate has its own scale, so a format may appear only once in `formats`
+ * (MOFQ_ERR_UNSUPPORTED otherwise).  mse_out: device, n floats.  workspace as for mofq_tensor_error.
  */
 int mofq_tensor_error_scaled(const mofq_tensor *x, const int32_t *formats, int n, const float *scales_in, float *mse_out,
                              void *workspace, size_t workspace_bytes, void *stream);
@@ -183,6 +200,9 @@ int mofq_tensor_error_scaled(const mofq_tensor *x, const int32_t *formats, int n
  * mofq_layer_output_error - error of the layer output Y = X W^T when its inputs are quantised
  * (Section 3.2 layer analysis; Algorithm 1 `compute_error` with the layer output metric).
  * is_w_only: Yq = X dq(W)^T; otherwise Yq = dq(X) dq(W)^T with the same format for both tensors.
+ * Scales: the paper's (Section 3.2) and the only ones this metric takes: cfg->w_gran = MOFQ_PER_CHANNEL and, unless
+ * is_w_only, cfg->a_gran = MOFQ_PER_TENSOR, so that the scales factor out of the contraction; anything else is
+ * MOFQ_ERR_UNSUPPORTED, as are fp16 activations with bf16 weights (no exact common 16-bit operand type).
  *   mse_out, nsr_out   device, cfg->n_candidates floats each, caller's order
  *   workspace          at least mofq_workspace_bytes(L, 1, cfg); first int32 = status bits
  */
@@ -255,7 +275,9 @@ int mofq_select_formats_host(const mofq_layer *layers_host_data, int n_layers, c
  *     more scratch than the built-in array holds, are refused with MOFQ_ERR_SCRATCH_LIMIT and
  *     nothing is enqueued.  Use mofq_tensor_error with your own workspace for those.
  *   - The first call on each device looks up the device address of the array (a one-time
- *     set-up, done with that device current).  Make that first call outside any stream capture.
+ *     set-up, done with that device current) and keeps it for the life of the process.  Make
+ *     that first call outside any stream capture.  A device that is reset (cudaDeviceReset) after
+ *     that first call must not use this entry point again: the kept address would be stale.
  *   - All calls on a device share the one array, and it still holds the previous call's data when
  *     the next call starts; each call clears the words that must start at zero.  Two calls that
  *     can run on the GPU at the same time (different streams, or different host threads without

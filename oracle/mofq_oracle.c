@@ -30,15 +30,6 @@
 #include <omp.h>
 #endif
 
-/* ORC_MUTATION (default 0 = none) plants one deliberate mistake; it exists only so that a test can show that the
- * pins reject a wrong oracle.  1: FP ties away from zero  2: E4M3 top code treated as a value (max 480)
- * 3: scale uses Q+1  4: MSE divides by rows instead of rows*cols  5: layer output uses W^T indexing swapped
- * 6: selection uses <=  7: subnormals flushed (no gradual underflow)  8: INT ties away from zero
- * 9: blocks numbered group-major instead of row-major */
-#ifndef ORC_MUTATION
-#define ORC_MUTATION 0
-#endif
-
 /* ---- enumerations (values are part of the oracle's own interface) -------------------------- */
 enum { ORC_INT4 = 0, ORC_INT8 = 1, ORC_FP4_E2M1 = 2, ORC_FP4_E2M1_IEEE = 3, ORC_FP8_E4M3 = 4, ORC_FP8_E5M2 = 5 };
 enum { ORC_PER_TENSOR = 0, ORC_PER_CHANNEL = 1, ORC_PER_GROUP = 2 };
@@ -152,9 +143,7 @@ double orc_decode(int fmt, int code)
     int m = code & ((1 << f.M) - 1);
     int emax_field = (1 << f.E) - 1;
     if (f.top_reserved == 1 && e == emax_field) return NAN;
-#if ORC_MUTATION != 2
     if (f.top_reserved == 2 && e == emax_field && m == (1 << f.M) - 1) return NAN;
-#endif
     double v = (e == 0) ? ldexp((double)m / (double)(1 << f.M), 1 - f.bias)
                         : ldexp(1.0 + (double)m / (double)(1 << f.M), e - f.bias);
     return s ? -v : v;
@@ -202,13 +191,7 @@ int orc_encode_fp_arith(int fmt, float t, int negative)
         (void)frexp(a, &ex);
         int e = ex - 1;
         if (e < 1 - f.bias) e = 1 - f.bias;
-#if ORC_MUTATION == 7
-        if (a < ldexp(1.0, 1 - f.bias)) a = 0.0;
-#endif
         double m = nearbyint(ldexp(a, f.M - e));     /* RNE: default rounding mode */
-#if ORC_MUTATION == 1
-        m = floor(ldexp(a, f.M - e) + 0.5);
-#endif
         v = ldexp(m, e - f.M);
         if (v > f.fmt_max) v = f.fmt_max;
     }
@@ -240,9 +223,6 @@ int orc_encode_int(int fmt, float t)
     fmt_t f;
     if (fmt_lookup(fmt, &f) || f.is_fp) return -1;
     double q = nearbyint((double)t);
-#if ORC_MUTATION == 8
-    q = t >= 0 ? floor((double)t + 0.5) : ceil((double)t - 0.5);
-#endif
     double lo = -f.fmt_max - 1.0, hi = f.fmt_max;
     if (q < lo) q = lo;
     if (q > hi) q = hi;
@@ -260,9 +240,6 @@ void orc_scale_from_absmax(int fmt, float absmax, float *scale, float *inv)
     fmt_t f;
     fmt_lookup(fmt, &f);
     float Q = (float)f.fmt_max;
-#if ORC_MUTATION == 3
-    Q += 1.0f;
-#endif
     if (absmax == 0.0f) { *scale = 1.0f; *inv = 1.0f; return; }
     *scale = absmax / Q;
     *inv = Q / absmax;
@@ -371,11 +348,7 @@ int orc_tensor_mse(const uint16_t *x, int dtype, int64_t rows, int64_t cols, int
     double sse;
     int rc = orc_quantize(x, dtype, rows, cols, ld, fmt, gran, group, NULL, NULL, NULL, NULL, &sse);
     if (rc) return rc;
-#if ORC_MUTATION == 4
-    *mse_out = sse / (double)rows;
-#else
     *mse_out = (rows > 0 && cols > 0) ? sse / (double)(rows * cols) : 0.0;
-#endif
     return 0;
 }
 
@@ -428,11 +401,7 @@ int orc_layer_output_error(const uint16_t *X, int dtype_x, int64_t T, int64_t ld
             for (int64_t o = 0; o < out; ++o) {
                 double y = 0.0, yq = 0.0;
                 for (int64_t i = 0; i < in; ++i) {
-#if ORC_MUTATION == 5
-                    y += Xd[t * in + i] * Wd[(o * in + i) % (out * in) == 0 ? 0 : ((i * out + o) % (out * in))];
-#else
                     y += Xd[t * in + i] * Wd[o * in + i];
-#endif
                     yq += Xq[t * in + i] * Wq[o * in + i];
                 }
                 noise += (y - yq) * (y - yq);
@@ -451,11 +420,7 @@ int orc_select(const double *errors, int n)
     double min_error = INFINITY;
     int best = -1;
     for (int i = 0; i < n; ++i)
-#if ORC_MUTATION == 6
-        if (errors[i] <= min_error) { min_error = errors[i]; best = i; }
-#else
         if (errors[i] < min_error) { min_error = errors[i]; best = i; }
-#endif
     return best;
 }
 
@@ -494,11 +459,7 @@ int orc_block_sse(const uint16_t *x, int dtype, int64_t rows, int64_t cols, int6
                 double e = (double)xv - orc_decode(fmt, code) * (double)scale;
                 sse += e * e;
             }
-#if ORC_MUTATION == 9
-            sse_out[b * rows + r] = sse;
-#else
             sse_out[r * per_row + b] = sse;
-#endif
         }
     return 0;
 }

@@ -308,6 +308,12 @@ int mofq_tensor_error_scaled(const mofq_tensor *x, const int32_t *formats, int n
     CandSet cs;
     int perm[MOFQ_MAX_CAND], nc, fp_formats[2];
     if (int rc = build_candset(formats, n, d0.bits, &cs, perm, &nc, fp_formats)) return rc;
+    // every candidate carries a scale of its own, so a format may appear only once (a repeat would share a kernel slot,
+    // and with it one scale)
+    for (int i = 0; i < n; ++i)
+        for (int k = 0; k < i; ++k)
+            if (formats[i] == formats[k]) return MOFQ_ERR_UNSUPPORTED;
+    if (x->cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
     if (int rc = check_ws(workspace, workspace_bytes, mofq_tensor_workspace_bytes(x))) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
@@ -337,6 +343,7 @@ int mofq_layer_output_error(const mofq_layer *L, const mofq_config *cfg, float *
     mofq_config c = *cfg;
     c.metric = MOFQ_LAYER_OUTPUT_MSE;
     c.w_gran2 = MOFQ_GRAN_NONE;
+    if (int rc = layer_metric_check(*L, &c)) return rc;
     if (int rc = check_ws(workspace, workspace_bytes, mofq_workspace_bytes(L, 1, &c))) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
@@ -363,6 +370,7 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
         if (cfg->metric == MOFQ_LAYER_OUTPUT_MSE) {
             if (int rc = check_tensor(&layers[i].X)) return rc;
             if (layers[i].X.cols != layers[i].W.cols) return MOFQ_ERR_INVALID_ARG;
+            if (int rc = layer_metric_check(layers[i], cfg)) return rc;
         }
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);

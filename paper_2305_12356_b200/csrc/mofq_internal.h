@@ -143,6 +143,8 @@ int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void
 // layer-output metric (mofq_layer.cu): extra workspace beyond the scoring workspace, and one layer's run.
 // Exactly one of `res` (selection record) or `mse_out`/`nsr_out` (raw errors, caller's order) is given.
 size_t layer_metric_ws_bytes(const mofq_layer *layers, int n_layers, const mofq_config *cfg);
+// the argument combinations layer_metric_run refuses (host-side checks only; nothing is enqueued)
+int layer_metric_check(const mofq_layer &L, const mofq_config *cfg);
 int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *res, float *mse_out, float *nsr_out,
                      void *workspace, size_t workspace_bytes, cudaStream_t st);
 

@@ -31,14 +31,8 @@
 namespace mofq {
 namespace {
 
-#ifndef MOFQ_MT_STAGES
-#define MOFQ_MT_STAGES 2
-#endif
-#ifndef MOFQ_MT_CTAS_PER_SM
-#define MOFQ_MT_CTAS_PER_SM 3
-#endif
-constexpr int kStages = MOFQ_MT_STAGES;
-constexpr int kCtasPerSm = MOFQ_MT_CTAS_PER_SM;   // kStages * kTileBytes * kCtasPerSm must fit one SM's shared memory
+constexpr int kStages = 2;
+constexpr int kCtasPerSm = 3;   // kStages * kTileBytes * kCtasPerSm must fit one SM's shared memory
 constexpr int kTileBytes = 32768;
 constexpr int kConsumerWarps = 4;
 constexpr int kConsumers = kConsumerWarps * 32;

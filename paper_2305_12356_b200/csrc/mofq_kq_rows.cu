@@ -11,8 +11,8 @@
 //   pass 2 of a tile: scales from rowmax (and segmax when group scales are scored too), then every candidate's
 //                     squared error from one walk over the segment's 16-byte chunks.
 // Pass 1 runs one tile AHEAD of pass 2, so the "every warp has finished pass 1 of this tile" barrier has normally
-// completed long before anyone waits on it, and with three or more stages the copy of the tile after that is in
-// flight meanwhile.  Rounds are dealt to the warps round-robin over the CTA's whole tile sequence (a fixed function
+// completed long before anyone waits on it, and the copies of the tiles after that are in flight meanwhile (the ring
+// holds three to six tiles, depending on the layer's tile size).  Rounds are dealt to the warps round-robin over the CTA's whole tile sequence (a fixed function
 // of the launch geometry, so sums are formed in the same order on every run), which keeps all lanes busy whatever
 // the number of segments per tile.  Per (layer, CTA, warp) partial sums go to the workspace and are added in slot
 // order: by a small finalize kernel for a layer list, by the last CTA to finish for a single tensor.
@@ -37,13 +37,15 @@ namespace {
 using namespace kqmath;
 using namespace kqpipe;
 
-constexpr int kRmConsumerWarps = 8;
-constexpr int kRmThreads = (kRmConsumerWarps + 1) * 32;    // + the producer warp
-constexpr int kRmTileCap = 72 * 1024;                      // most bytes of one tile
-constexpr int kRmStageMeta = 2 * (kRmTileCap / 256) * 4;   // per stage: abs-max pattern of every segment and of every row
-constexpr int kRmSmemBudget = 3 * (kRmTileCap + kRmStageMeta) + 1024;   // three stages of the largest tile (222 KB of the SM's 227)
-constexpr int kRmMaxStages = 8;
+constexpr int kRmConsumerWarps = 12;                       // warps 0..11: pass 2 (scoring), three per scheduler
+constexpr int kRmScoutWarps = 4;                           // warps 12..15: pass 1 (abs-max), one per scheduler
+constexpr int kRmThreads = (kRmConsumerWarps + kRmScoutWarps + 1) * 32;    // + the producer warp
+constexpr int kRmTileCap = 70 * 1024;                      // most bytes of one tile (two rows of 17920 fp16)
 constexpr int kRmMaxSeg = kRmTileCap / 256;                // segments (= most rows) of one tile
+constexpr int kRmSlots = 6;                                // tiles in flight: barrier sets and per-tile tables
+constexpr int kRmRingBytes = 212 * 1024;                   // shared-memory ring: 3 tiles of 70 KB, 5 of 40 KB, 6 of <= 35 KB
+constexpr int kRmSlotMeta = 2 * kRmMaxSeg * 4;             // per slot: abs-max pattern of every segment and of every row
+constexpr int kRmSmemBytes = kRmRingBytes + kRmSlots * kRmSlotMeta + 1024;   // + slack to align the ring
 
 // One layer of the work table (device memory, or inline in the parameters for a single tensor).
 struct RmLayer {
@@ -57,18 +59,19 @@ struct RmLayer {
     int rows_per_tile;
     int segs_per_row;
     uint32_t row_magic;       // segment index -> row within the tile: (q * row_magic) >> 16
+    int stage_bytes, stages;  // how this layer's tiles divide the ring
     int first_cta, n_slots, slot_off, pad;
 };
 
 struct RmTileInfo {           // what the producer publishes with each tile
     int nseg, nrows, layer;
-    uint32_t row_magic;
+    uint32_t row_magic, smem_off;
 };
 
 struct RmParams {
     const RmLayer *layers;    // nullptr: `one` is the only layer
     RmLayer one;
-    int n_layers, stages, stage_bytes, grp_first;
+    int n_layers, grp_first;
     long long total_tiles, total_w;
     RowQ rq;
     double *partials;         // [slot][kMaxAcc]
@@ -107,6 +110,9 @@ __device__ __forceinline__ int find_layer(const RmLayer *layers, int n, long lon
     return lo;
 }
 
+// The CTA's tiles are numbered it = 0, 1, ...; tile `it` uses barrier set and tables it % kRmSlots, in phase it / kRmSlots.
+__device__ __forceinline__ uint32_t slot_parity(int it) { return (uint32_t)(it / kRmSlots) & 1u; }
+
 template <int DT, int NI, int K0, int K1, bool GRP>
 __global__ void __launch_bounds__(kRmThreads, 1)
 kq_score_rows_mt(const __grid_constant__ RmParams p)
@@ -115,22 +121,22 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
     constexpr int NC = S::NC;
     constexpr int NA = NC * (GRP ? 2 : 1);
     extern __shared__ __align__(16) unsigned char smem[];   // aligned by hand below
-    __shared__ __align__(8) uint64_t full_bar[kRmMaxStages], empty_bar[kRmMaxStages], row_bar[kRmMaxStages];
-    __shared__ RmTileInfo tinfo[kRmMaxStages];
+    __shared__ __align__(8) uint64_t full_bar[kRmSlots], empty_bar[kRmSlots], row_bar[kRmSlots];
+    __shared__ RmTileInfo tinfo[kRmSlots];
     __shared__ int err;
     __shared__ int is_last;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (smem_u32(smem) + 1023u) & ~1023u;
     unsigned char *const smem_al = smem + (smem_base - smem_u32(smem));
-    // behind the ring: per stage the segments' abs-max patterns and the rows' abs-max patterns
-    uint32_t *const segmax = reinterpret_cast<uint32_t *>(smem_al + (size_t)p.stages * p.stage_bytes);
-    uint32_t *const rowmax = segmax + p.stages * kRmMaxSeg;
+    // behind the ring: per slot the segments' abs-max patterns and the rows' abs-max patterns
+    uint32_t *const segmax = reinterpret_cast<uint32_t *>(smem_al + kRmRingBytes);
+    uint32_t *const rowmax = segmax + kRmSlots * kRmMaxSeg;
     const RmLayer *const layers = p.layers ? p.layers : &p.one;
     if (tid == 0) {
-        for (int s = 0; s < p.stages; ++s) {
+        for (int s = 0; s < kRmSlots; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kRmConsumerWarps);
-            mbar_init(&row_bar[s], kRmConsumerWarps);
+            mbar_init(&row_bar[s], kRmScoutWarps);
         }
         err = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -144,64 +150,130 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
     for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
     int status = 0;
 
-    if (warp == kRmConsumerWarps) {
-        // ---------------- producer warp: lane 0 issues the copies, all lanes clear the stage's row maxima ----------------
+    if (warp == kRmConsumerWarps + kRmScoutWarps) {
+        // ---------------- producer warp: lane 0 issues the copies, all lanes clear the tile's row maxima ----------------
+        // A layer's tiles cycle through `stages` (>= 3) equal parts of the ring (its own division: small tiles get
+        // more parts).  Tiles are released in order, so "tile it - stages has been released" frees the part tile `it`
+        // takes.  A new layer's first tile does not wait for the last tile of the layer before it (that would leave the
+        // ring empty at every change of layer): it goes to a part of the new division that does not touch that tile's
+        // bytes, and the new division's other parts are used once that tile, too, has been released.
         int layer = n_it > 0 ? find_layer(layers, p.n_layers, t_begin) : 0;
         RmLayer L = layers[layer];
-        int s = 0;
-        uint32_t ph = 0;
+        int run = 0;          // tiles issued under the current division of the ring
+        int first_part = 0;   // part of the current division that its first tile took
+        uint32_t prev_off = 0, prev_bytes = 0;   // where the tile issued last sits
         bool ok = true;
         for (int it = 0; it < n_it && ok; ++it) {
             const long long t = t_begin + it;
-            while (t >= L.tile_begin + L.n_tiles) L = layers[++layer];
-            ok = mbar_wait(&empty_bar[s], ph ^ 1u, &err);      // every consumer warp has left the stage's previous tile
+            if (t >= L.tile_begin + L.n_tiles) {
+                while (t >= L.tile_begin + L.n_tiles) L = layers[++layer];
+                run = 0;
+                first_part = 0;
+                while (first_part + 1 < L.stages && (uint32_t)first_part * (uint32_t)L.stage_bytes < prev_off + prev_bytes &&
+                       (uint32_t)(first_part + 1) * (uint32_t)L.stage_bytes > prev_off)
+                    ++first_part;
+            }
+            // The tiles whose release frees this tile's place.  The groups release their tiles in any order, so every
+            // tile that must be gone is waited for by name: the one that had this tile's barrier set and tables, and
+            // then either the tile that had its part of the ring or, after a change of layer, every tile of the old
+            // division (all but the last one before the new division's first tile, the last one too after that).
+            if (it >= kRmSlots) ok = mbar_wait(&empty_bar[it % kRmSlots], slot_parity(it - kRmSlots), &err);
+            if (run == 0) {
+                for (int k = max(0, it - kRmSlots + 1); k <= it - 2 && ok; ++k) ok = mbar_wait(&empty_bar[k % kRmSlots], slot_parity(k), &err);
+            } else {
+                const int need = run < L.stages ? it - run - 1 : it - L.stages;
+                if (need >= 0 && ok) ok = mbar_wait(&empty_bar[need % kRmSlots], slot_parity(need), &err);
+            }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
+            const int slot = it % kRmSlots;
             const long long r0 = (t - L.tile_begin) * L.rows_per_tile;
             const int nr = (int)min((long long)L.rows_per_tile, L.rows - r0);
-            for (int r = lane; r < nr; r += 32) rowmax[s * kRmMaxSeg + r] = 0;
+            for (int r = lane; r < nr; r += 32) rowmax[slot * kRmMaxSeg + r] = 0;
             __syncwarp();
+            const uint32_t off = (uint32_t)((first_part + run) % L.stages) * (uint32_t)L.stage_bytes;
+            prev_off = off;
+            prev_bytes = (uint32_t)L.stage_bytes;
             if (lane == 0) {
-                tinfo[s].nseg = nr * L.segs_per_row;
-                tinfo[s].nrows = nr;
-                tinfo[s].layer = layer;
-                tinfo[s].row_magic = L.row_magic;
+                tinfo[slot].nseg = nr * L.segs_per_row;
+                tinfo[slot].nrows = nr;
+                tinfo[slot].layer = layer;
+                tinfo[slot].row_magic = L.row_magic;
+                tinfo[slot].smem_off = off;
                 const uint32_t row_bytes = (uint32_t)L.cols * 2u;
-                mbar_expect_tx(&full_bar[s], (uint32_t)nr * row_bytes);   // (release: the stores above are visible to the waiters)
-                unsigned char *dst = smem_al + (size_t)s * p.stage_bytes;
+                mbar_expect_tx(&full_bar[slot], (uint32_t)nr * row_bytes);   // (release: the stores above are visible to the waiters)
+                unsigned char *dst = smem_al + off;
                 if (L.ld == L.cols) {
-                    bulk_load(dst, L.x + r0 * L.ld, (uint32_t)nr * row_bytes, &full_bar[s]);
+                    bulk_load(dst, L.x + r0 * L.ld, (uint32_t)nr * row_bytes, &full_bar[slot]);
                 } else {
-                    for (int r = 0; r < nr; ++r) bulk_load(dst + (size_t)r * row_bytes, L.x + (r0 + r) * L.ld, row_bytes, &full_bar[s]);
+                    for (int r = 0; r < nr; ++r) bulk_load(dst + (size_t)r * row_bytes, L.x + (r0 + r) * L.ld, row_bytes, &full_bar[slot]);
                 }
             }
-            if (++s == p.stages) {
-                s = 0;
-                ph ^= 1u;
-            }
+            ++run;
         }
         if (!ok && lane == 0) {
             // give copies already issued a bounded chance to land before the shared memory is released
-            for (int k = 0; k < p.stages; ++k) {
+            for (int k = 0; k < kRmSlots; ++k) {
                 const long long t0 = clock64();
                 while (!mbar_try_wait(&full_bar[k], 0) && !mbar_try_wait(&full_bar[k], 1) && clock64() - t0 < kWaitCycles) {}
             }
             atomicOr(p.timeout, MOFQ_STATUS_TIMEOUT);
         }
+    } else if (warp >= kRmConsumerWarps) {
+        // ---------------- scout warps: pass 1 of every tile as soon as it has landed ----------------
+        // The maxima do not depend on who forms them or in which order, and this pass is bound by the latency of its
+        // chain of maxima, not by issue slots: one light warp per scheduler does it for all, so that the scoring
+        // warps never wait for one another's pass 1.
+        const int sid = warp - kRmConsumerWarps;
+        bool ok = true;
+        for (int it = 0; it < n_it && ok; ++it) {
+            const int slot = it % kRmSlots;
+            ok = mbar_wait(&full_bar[slot], slot_parity(it), &err);
+            if (!ok) break;
+            const RmTileInfo ti = tinfo[slot];
+            const int rounds = (ti.nseg + 31) >> 5;
+            const uint32_t tile = smem_base + ti.smem_off;
+            for (int r = (sid + it) % kRmScoutWarps; r < rounds; r += kRmScoutWarps) {   // rotated: no scout gets the extra round every time
+                const int q = r * 32 + lane;
+                const bool live = q < ti.nseg;
+                uint32_t m16 = 0;
+                if (live) {
+                    const uint32_t a0 = tile + (uint32_t)q * 256u + (uint32_t)((q & 15) << 4);
+                    uint32_t m[4] = {0, 0, 0, 0};   // four independent chains
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) m[k & 3] = absmax_chunk<DT>(lds128(a0 ^ (uint32_t)(k << 4)), m[k & 3]);
+                    m16 = max(max(fold16(m[0]), fold16(m[1])), max(fold16(m[2]), fold16(m[3])));
+                    segmax[slot * kRmMaxSeg + q] = m16;
+                }
+                // the round's segments lie in one or two rows unless rows are shorter than a round: one shared-memory
+                // update per row instead of one per lane
+                const uint32_t row = ((uint32_t)min(q, ti.nseg - 1) * ti.row_magic) >> 16;
+                const uint32_t row0 = __shfl_sync(0xffffffffu, row, 0);
+                if (__all_sync(0xffffffffu, row - row0 <= 1u)) {
+                    const uint32_t m0 = __reduce_max_sync(0xffffffffu, row == row0 ? m16 : 0u);
+                    const uint32_t m1 = __reduce_max_sync(0xffffffffu, row != row0 ? m16 : 0u);
+                    if (lane == 0) {
+                        atomicMax(&rowmax[slot * kRmMaxSeg + row0], m0);
+                        if (m1) atomicMax(&rowmax[slot * kRmMaxSeg + row0 + 1], m1);
+                    }
+                } else if (live) {
+                    atomicMax(&rowmax[slot * kRmMaxSeg + row], m16);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&row_bar[slot]);     // (release: the maxima above are visible to whoever waits)
+        }
+        if (!ok && lane == 0) atomicOr(p.timeout, MOFQ_STATUS_TIMEOUT);
     } else {
-        // ---------------- consumer warps ----------------
-        // rounds of the CTA's tile sequence are numbered consecutively; warp w takes the rounds congruent to w.
-        // off1 / off2: this warp's first round inside the tile that pass 1 / pass 2 takes next.
-        int off1 = warp, off2 = warp;
-        int s1 = 0, s2 = 0;
-        uint32_t ph1 = 0, ph2 = 0;
+        // ---------------- consumer warps: pass 2 ----------------
+        // The rounds of the CTA's tile sequence are numbered consecutively and warp w takes the rounds congruent to w:
+        // a fixed function of the launch geometry, so sums are formed in the same order on every run.  A warp waits
+        // only for the scouts' pass 1 of the tile at hand; the warps drift apart by as many tiles as the ring holds,
+        // which evens out the rounds that do not divide among them tile by tile.
+        int off2 = warp;      // this warp's first round inside the next tile
         int cur_layer = -1;
         RmLayer L = layers[0];
 
-        auto advance = [](int &off, int rounds) {
-            off -= rounds % kRmConsumerWarps;
-            if (off < 0) off += kRmConsumerWarps;
-        };
         auto flush = [&]() __attribute__((always_inline)) {
             // this warp's partial sums of the finished layer -> its slot; the slots are added in order later
 #pragma unroll
@@ -219,61 +291,25 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
             for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
             status = 0;
         };
-        // pass 1 of the next tile in line: abs-max of this warp's segments
-        auto pass1 = [&]() __attribute__((always_inline)) -> bool {
-            const int s = s1;
-            const bool ok = mbar_wait(&full_bar[s], ph1, &err);
-            if (++s1 == p.stages) {
-                s1 = 0;
-                ph1 ^= 1u;
-            }
-            if (ok) {
-                const RmTileInfo ti = tinfo[s];
-                const int rounds = (ti.nseg + 31) >> 5;
-                const uint32_t tile = smem_base + (uint32_t)s * (uint32_t)p.stage_bytes;
-                for (int r = off1; r < rounds; r += kRmConsumerWarps) {
-                    const int q = r * 32 + lane;
-                    if (q < ti.nseg) {
-                        const uint32_t a0 = tile + (uint32_t)q * 256u + (uint32_t)((q & 15) << 4);
-                        uint32_t m = 0;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) m = absmax_chunk<DT>(lds128(a0 ^ (uint32_t)(j << 4)), m);
-                        const uint32_t m16 = fold16(m);
-                        segmax[s * kRmMaxSeg + q] = m16;
-                        atomicMax(&rowmax[s * kRmMaxSeg + ((q * ti.row_magic) >> 16)], m16);
-                    }
-                }
-                advance(off1, rounds);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&row_bar[s]);     // arrives even after a failed wait: nobody is left waiting for this warp
-            return ok;
-        };
 
         bool ok = true;
-        if (n_it > 0) ok = pass1();
         for (int it = 0; it < n_it; ++it) {
-            if (it + 1 < n_it) ok = pass1() && ok;
-            const int s = s2;
-            ok = mbar_wait(&row_bar[s], ph2, &err) && ok;   // every warp has finished pass 1 of this tile
-            if (++s2 == p.stages) {
-                s2 = 0;
-                ph2 ^= 1u;
-            }
+            const int slot = it % kRmSlots;
+            ok = mbar_wait(&row_bar[slot], slot_parity(it), &err) && ok;   // the scouts have finished pass 1 of this tile
             if (ok) {
-                const RmTileInfo ti = tinfo[s];
+                const RmTileInfo ti = tinfo[slot];
                 if (ti.layer != cur_layer) {
                     if (cur_layer >= 0) flush();
                     cur_layer = ti.layer;
                     L = layers[cur_layer];
                 }
                 const int rounds = (ti.nseg + 31) >> 5;
-                const uint32_t tile = smem_base + (uint32_t)s * (uint32_t)p.stage_bytes;
+                const uint32_t tile = smem_base + ti.smem_off;
                 for (int r = off2; r < rounds; r += kRmConsumerWarps) {
                     const int q = r * 32 + lane;
                     if (q < ti.nseg) {
                         const uint32_t a0 = tile + (uint32_t)q * 256u + (uint32_t)((q & 15) << 4);
-                        const uint32_t rm = rowmax[s * kRmMaxSeg + ((q * ti.row_magic) >> 16)];
+                        const uint32_t rm = rowmax[slot * kRmMaxSeg + ((q * ti.row_magic) >> 16)];
                         if (mag16_nonfinite<DT>(rm)) status |= MOFQ_STATUS_NONFINITE_INPUT;
                         Sc<NC> sc;
                         S s_c, s_g;
@@ -284,7 +320,7 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
                         }
                         s_c.begin(sc);
                         if (GRP) {
-                            const uint32_t gm = segmax[s * kRmMaxSeg + q];
+                            const uint32_t gm = segmax[slot * kRmMaxSeg + q];
 #pragma unroll
                             for (int j = 0; j < NC; ++j) {
                                 if (DT == MOFQ_F16) scale_pair_fast(mag16_to_float<DT>(gm), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
@@ -314,10 +350,11 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
                         }
                     }
                 }
-                advance(off2, rounds);
+                off2 -= rounds % kRmConsumerWarps;
+                if (off2 < 0) off2 += kRmConsumerWarps;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[s]);
+            if (lane == 0) mbar_arrive(&empty_bar[slot]);
         }
         if (cur_layer >= 0) flush();
         if (!ok && lane == 0) atomicOr(p.timeout, MOFQ_STATUS_TIMEOUT);   // a wait expired: the sums are incomplete
@@ -477,6 +514,8 @@ bool describe_layer(const mofq_tensor &W, RmLayer *L, bool single = false)
     L->rows_per_tile = rows_per_tile(W.rows, (int)W.cols, single);
     L->n_tiles = (W.rows + L->rows_per_tile - 1) / L->rows_per_tile;
     L->inv_n = 1.0 / ((double)W.rows * (double)W.cols);
+    L->stage_bytes = (L->rows_per_tile * (int)W.cols * 2 + 1023) & ~1023;
+    L->stages = std::min(kRmSlots, kRmRingBytes / L->stage_bytes);   // >= 3: a tile is at most a third of the ring
     // q / segs_per_row for q < kRmMaxSeg through a multiply and a shift (checked here for every q)
     L->row_magic = (65536u + (uint32_t)L->segs_per_row - 1u) / (uint32_t)L->segs_per_row;
     for (uint32_t q = 0; q < (uint32_t)kRmMaxSeg; ++q)
@@ -487,14 +526,13 @@ bool describe_layer(const mofq_tensor &W, RmLayer *L, bool single = false)
 struct RmPlan {
     std::vector<RmLayer> table;
     long long total_tiles = 0, total_w = 0;
-    int grid = 1, stages = 3, stage_bytes = 0;
+    int grid = 1;
     long long slots = 0;
 };
 
 bool make_plan(const mofq_tensor *const *tensors, int n, RmPlan *plan)
 {
     plan->table.resize((size_t)n);
-    int max_tile = 0;
     long long tiles = 0, w = 0;
     for (int i = 0; i < n; ++i) {
         RmLayer &L = plan->table[(size_t)i];
@@ -504,12 +542,9 @@ bool make_plan(const mofq_tensor *const *tensors, int n, RmPlan *plan)
         L.w_begin = w;
         tiles += L.n_tiles;
         w += L.n_tiles * L.rows_per_tile * L.segs_per_row;   // the last tile of a layer counts as a full one
-        max_tile = std::max(max_tile, L.rows_per_tile * L.cols * 2);
     }
     plan->total_tiles = tiles;
     plan->total_w = w;
-    plan->stage_bytes = (max_tile + 1023) & ~1023;
-    plan->stages = std::max(2, std::min(kRmMaxStages, (kRmSmemBudget - 1024) / (plan->stage_bytes + kRmStageMeta)));
     // every CTA's share of the weight holds at least one tile begin, so that no CTA between two others is idle
     const long long by_weight = std::max<long long>(1, w / kRmMaxSeg);
     plan->grid = (int)std::max<long long>(1, std::min<long long>(std::min<long long>(sm_count(), tiles), by_weight));
@@ -532,15 +567,10 @@ bool make_plan(const mofq_tensor *const *tensors, int n, RmPlan *plan)
     return true;
 }
 
-size_t smem_bytes(const RmPlan &plan)
-{
-    return (size_t)plan.stages * (plan.stage_bytes + kRmStageMeta) + 1024;   // + slack to align the tiles
-}
-
 template <typename K>
 int launch_kernel(K kernel, const RmPlan &plan, const RmParams &p, cudaStream_t st)
 {
-    const size_t smem = smem_bytes(plan);
+    const size_t smem = kRmSmemBytes;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
         (void)cudaGetLastError();
         return MOFQ_ERR_CUDA;
@@ -553,8 +583,6 @@ int launch_kernel(K kernel, const RmPlan &plan, const RmParams &p, cudaStream_t 
 int launch_plan(const RmPlan &plan, RmParams &p, int dtype, const CandSet &cs, const int *fp_formats, bool has_grp, cudaStream_t st)
 {
     p.n_layers = (int)plan.table.size();
-    p.stages = plan.stages;
-    p.stage_bytes = plan.stage_bytes;
     p.total_tiles = plan.total_tiles;
     p.total_w = plan.total_w;
     p.rq = candset_rowq(cs);

@@ -20,7 +20,6 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
-#include <cstdlib>
 #include <type_traits>
 
 #include "mofq_internal.h"
@@ -696,8 +695,7 @@ int run_gemm_n(int n, const void *const *a, long long a_rows, const long long *a
     const int npair = std::max(1, nsm / 2);
     const double c128 = (double)((t128 + nsm - 1) / nsm) * 1.0, c256 = (double)((t256 + nsm - 1) / nsm) * 1.5;
     const double cpair = (double)((tpair + npair - 1) / npair) * 1.0;
-    const bool force_single = getenv("MOFQ_GEMM_SINGLE_CTA") != nullptr;
-    const int cg = (!force_single && cpair < std::min(c128, c256)) ? 2 : 1;
+    const int cg = cpair < std::min(c128, c256) ? 2 : 1;
     const int bn = cg == 2 ? 256 : (c256 < c128 ? 256 : 128);
     GemmMaps maps;
     GemmParams p{};
@@ -797,8 +795,7 @@ size_t layer_metric_ws_bytes(const mofq_layer *layers, int n_layers, const mofq_
     return need;
 }
 
-int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *res, float *mse_out, float *nsr_out,
-                     void *workspace, size_t workspace_bytes, cudaStream_t st)
+int layer_metric_check(const mofq_layer &L, const mofq_config *cfg)
 {
     const mofq_tensor &W = L.W, &X = L.X;
     if (X.cols != W.cols) return MOFQ_ERR_INVALID_ARG;
@@ -806,11 +803,22 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
     if (!cfg->is_w_only && cfg->a_gran != MOFQ_PER_TENSOR) return MOFQ_ERR_UNSUPPORTED;
     if (X.dtype == MOFQ_F16 && W.dtype == MOFQ_BF16) return MOFQ_ERR_UNSUPPORTED;    // no exact common 16-bit operand type
     if (W.rows > 0x7fffffffLL || X.rows > 0x7fffffffLL || W.cols > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
-    FmtDesc fd[MOFQ_MAX_CAND];
+    if (!cfg->is_w_only && cfg->bit_width == 8 && W.cols * 2 > 200 * 1024) return MOFQ_ERR_UNSUPPORTED;  // the code emission stages a weight row in shared memory
     for (int i = 0; i < cfg->n_candidates; ++i) {
-        if (!describe_format(cfg->candidates[i], &fd[i])) return MOFQ_ERR_INVALID_ARG;
-        if (fd[i].bits != cfg->bit_width) return MOFQ_ERR_UNSUPPORTED;
+        FmtDesc fd;
+        if (!describe_format(cfg->candidates[i], &fd)) return MOFQ_ERR_INVALID_ARG;
+        if (fd.bits != cfg->bit_width) return MOFQ_ERR_UNSUPPORTED;
     }
+    return MOFQ_OK;
+}
+
+int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *res, float *mse_out, float *nsr_out,
+                     void *workspace, size_t workspace_bytes, cudaStream_t st)
+{
+    const mofq_tensor &W = L.W, &X = L.X;
+    if (int rc = layer_metric_check(L, cfg)) return rc;
+    FmtDesc fd[MOFQ_MAX_CAND];
+    for (int i = 0; i < cfg->n_candidates; ++i) describe_format(cfg->candidates[i], &fd[i]);
     const long long T = X.rows, n_in = W.cols, n_out = W.rows;
     const LayerWs lw = layer_ws_layout(T, n_in, n_out);
     const size_t base_off = align256(score_ws_bytes());
