@@ -116,8 +116,7 @@ int check_config(const mofq_config *cfg)
 
 // tensor metric for one layer: enqueue the scoring of W and the record(s) for it
 int score_layer_tensor(const mofq_tensor &W, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
-                       const int *fp_formats, mofq_result *res, float *mse_out, void *ws, cudaStream_t st,
-                       bool after_own_launch = false /* the previous launch on st is the previous layer's scoring */)
+                       const int *fp_formats, mofq_result *res, float *mse_out, void *ws, cudaStream_t st)
 {
     if (int rc = check_tensor(&W)) return rc;
     if (int rc = check_gran(cfg->w_gran, cfg->w_group, W.cols)) return rc;
@@ -151,7 +150,6 @@ int score_layer_tensor(const mofq_tensor &W, const mofq_config *cfg, const CandS
     job.fin.nc = nc;
     std::memcpy(job.fin.perm, perm, sizeof(job.fin.perm));
     job.fin.inv_n = 1.0 / ((double)W.rows * (double)W.cols);
-    job.overlap_prev = after_own_launch;
     return launch_score(job, st);
 }
 
@@ -385,7 +383,7 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
     for (int i = 0; i < n_layers; ++i) {  // Algorithm 1: for layer in model.layers_to_quant
         int rc;
         if (cfg->metric == MOFQ_TENSOR_MSE)
-            rc = score_layer_tensor(layers[i].W, cfg, cs, perm, nc, fp_formats, results_out + (size_t)i * n_sets, nullptr, workspace, st, i > 0);
+            rc = score_layer_tensor(layers[i].W, cfg, cs, perm, nc, fp_formats, results_out + (size_t)i * n_sets, nullptr, workspace, st);
         else
             rc = layer_metric_run(layers[i], cfg, results_out + i, nullptr, nullptr, workspace, workspace_bytes, st);
         if (rc) return rc;

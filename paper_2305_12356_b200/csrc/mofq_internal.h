@@ -74,10 +74,6 @@ struct ScoreJob {
     Finalize fin;
     WsHeader *hdr;
     double *partials;          // kMaxSlots * kMaxAcc doubles
-    // The previous launch on the stream is a scoring launch of the same library call (the layer before this one):
-    // this launch may then start while that one drains.  Never set for the first launch of a call, whose
-    // predecessor on the stream is the caller's own work.
-    bool overlap_prev;
 };
 
 inline size_t score_ws_bytes() { return sizeof(WsHeader) + sizeof(double) * kMaxSlots * kMaxAcc; }

@@ -352,214 +352,6 @@ kq_select_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long 
     block_finish<NA>(dacc, status, hdr, partials, fin, red);
 }
 
-// ---- scoring kernel 2b: whole rows streamed through a shared-memory ring --------------------------------------
-// Per-channel scales (optionally group-128 scales from the same read) for rows that are a multiple of 128
-// elements.  A tile is `rows_per_tile` whole rows; one producer thread brings tiles in with bulk asynchronous
-// copies that complete on mbarriers (three stages, two for rows too long for that), the consumer threads own 128-element segments of the tile.
-// Pass 1: segment abs-max -> shared-memory max per row; pass 2: every segment is scored against its row's scales
-// (and its own group scales) from shared memory.  The two passes are software-pipelined: a consumer runs pass 1 of
-// tile i+1 before pass 2 of tile i, so the "all of tile i's pass 1 is done" barrier (an mbarrier the warps arrive
-// on) has normally completed long before anyone waits on it.  Chunk addresses are formed by XOR, as in the
-// multi-tensor kernel.  All waits are bounded; a consumer that gave up still arrives on every barrier, so nobody is
-// left waiting for it.
-constexpr int kRsMaxStages = 3;
-constexpr int kRsMaxRows = 8;
-constexpr int kRsMaxTileBytes = 49152;
-constexpr int kRsMaxConsumers = 256;
-
-struct RsParams {
-    const uint16_t *x;
-    long long rows, ld, n_tiles, tiles_per_cta;
-    int cols, rows_per_tile, segs_per_row, consumers, stage_bytes, stages, grp_first;
-    RowQ rq;
-};
-
-struct RsSeg {          // what a consumer carries from pass 1 to pass 2 of a tile: up to two segments
-    uint32_t a0[2];     // shared-memory address of the segment (with the lane's XOR offset); 0 = none
-    uint32_t segmax[2];
-    int row[2];
-};
-
-template <int DT, int NI, int K0, int K1, bool GRP>
-__global__ void __launch_bounds__(kRsMaxConsumers + 32)
-kq_score_rows_stream(const RsParams p, WsHeader *hdr, double *partials, Finalize fin)
-{
-    using namespace kqpipe;
-    using S = kqmath::Scorer<DT, NI, K0, K1, true>;      // scales are fixed over a segment: scaled accumulation
-    constexpr int NC = S::NC;
-    constexpr int NA = NC * (GRP ? 2 : 1);
-    extern __shared__ __align__(16) unsigned char smem[];   // aligned by hand below
-    __shared__ __align__(8) uint64_t full_bar[kRsMaxStages], empty_bar[kRsMaxStages], row_bar[2];
-    __shared__ uint32_t rowmax[8][kRsMaxRows];
-    __shared__ int err;
-    __shared__ double red[33 * NA];
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n_cw = p.consumers >> 5;
-    const uint32_t smem_base = (smem_u32(smem) + 1023u) & ~1023u;
-    unsigned char *const smem_al = smem + (smem_base - smem_u32(smem));
-    if (tid == 0) {
-        for (int s = 0; s < p.stages; ++s) {
-            mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], n_cw);
-        }
-        mbar_init(&row_bar[0], n_cw);
-        mbar_init(&row_bar[1], n_cw);
-        err = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (tid < 8 * kRsMaxRows) (&rowmax[0][0])[tid] = 0;
-    __syncthreads();
-    // Programmatic dependent launch: the next launch on the stream (the next layer's scoring) may start as soon as
-    // every block of this one is running, so its blocks fill the SMs this launch's tail leaves idle.  Its reads are
-    // of its own input only; it waits for this launch to complete (below) before touching the shared workspace.
-    asm volatile("griddepcontrol.launch_dependents;");
-    const long long t_begin = (long long)blockIdx.x * p.tiles_per_cta;
-    const long long t_end = min(t_begin + p.tiles_per_cta, p.n_tiles);
-    const int n_it = t_end > t_begin ? (int)(t_end - t_begin) : 0;
-    const uint32_t row_bytes = (uint32_t)p.cols * 2u;
-    double dacc[NA];
-#pragma unroll
-    for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
-    int status = 0;
-
-    if (warp == n_cw) {
-        // ---------------- producer ----------------
-        if (lane == 0) {
-            for (int it = 0; it < n_it; ++it) {
-                const long long t = t_begin + it;
-                const int s = it % p.stages;
-                const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
-                if (!mbar_wait(&empty_bar[s], ph ^ 1u, &err)) break;
-                const long long r0 = t * p.rows_per_tile;
-                const int nr = (int)min((long long)p.rows_per_tile, p.rows - r0);
-                mbar_expect_tx(&full_bar[s], (uint32_t)nr * row_bytes);
-                unsigned char *dst = smem_al + (size_t)s * p.stage_bytes;
-                if (p.ld == p.cols) {
-                    bulk_load(dst, p.x + r0 * p.ld, (uint32_t)nr * row_bytes, &full_bar[s]);
-                } else {
-                    for (int r = 0; r < nr; ++r) bulk_load(dst + (size_t)r * row_bytes, p.x + (r0 + r) * p.ld, row_bytes, &full_bar[s]);
-                }
-            }
-            if (err) {
-                // give copies already issued a bounded chance to land before the shared memory is released
-                for (int s = 0; s < p.stages; ++s) {
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(&full_bar[s], 0) && !mbar_try_wait(&full_bar[s], 1) && clock64() - t0 < kWaitCycles) {}
-                }
-                status |= MOFQ_STATUS_TIMEOUT;
-            }
-        }
-    } else {
-        // ---------------- consumers ----------------
-        // a thread's segments sit at the same place in every tile: row within the tile and byte offset, once
-        int seg_row[2];
-        uint32_t seg_off[2];
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            const int g = tid + k * p.consumers;
-            seg_row[k] = g / p.segs_per_row;
-            seg_off[k] = (uint32_t)seg_row[k] * row_bytes + (uint32_t)(g - seg_row[k] * p.segs_per_row) * 256u + (uint32_t)((tid & 15) << 4);
-        }
-        int s1 = 0;            // stage and phase of the tile pass 1 takes next
-        uint32_t ph1 = 0;
-        // pass 1 of tile `it`: abs-max of this thread's segments, folded into the tile's per-row maxima
-        auto pass1 = [&](int it, RsSeg &sg) {
-            const int s = s1;
-            const uint32_t ph = ph1;
-            if (++s1 == p.stages) {
-                s1 = 0;
-                ph1 ^= 1u;
-            }
-            const bool ok = mbar_wait(&full_bar[s], ph, &err);
-            const long long r0 = (t_begin + it) * p.rows_per_tile;
-            const int nr = (int)min((long long)p.rows_per_tile, p.rows - r0);
-            const int nseg = ok ? nr * p.segs_per_row : 0;
-            const uint32_t tile = smem_base + (uint32_t)s * (uint32_t)p.stage_bytes;
-            uint32_t *rmax = rowmax[it & 7];
-#pragma unroll
-            for (int k = 0; k < 2; ++k) {                // at most two segments per consumer (the host sizes the tile so)
-                const int g = tid + k * p.consumers;
-                sg.a0[k] = 0;
-                sg.segmax[k] = 0;
-                sg.row[k] = 0;
-                if (g < nseg) {
-                    sg.row[k] = seg_row[k];
-                    sg.a0[k] = tile + seg_off[k];
-                    uint32_t m = 0;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) m = kqmath::absmax_chunk<DT>(lds128(sg.a0[k] ^ (uint32_t)(j << 4)), m);
-                    sg.segmax[k] = fold16(m);
-                    atomicMax(&rmax[sg.row[k]], sg.segmax[k]);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&row_bar[it & 1]);
-        };
-        RsSeg cur, nxt;
-        if (n_it > 0) pass1(0, cur);
-        int s2 = 0;            // stage pass 2 releases next
-        for (int it = 0; it < n_it; ++it) {
-            if (it + 1 < n_it) pass1(it + 1, nxt);
-            const bool ok = mbar_wait(&row_bar[it & 1], (uint32_t)(it >> 1) & 1u, &err);   // every warp has finished pass 1 of this tile
-            // the buffer four tiles ahead: nobody is within three tiles of it on either side
-            if (tid < kRsMaxRows) rowmax[(it + 4) & 7][tid] = 0;
-            const uint32_t *rmax = rowmax[it & 7];
-#pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                if (ok && cur.a0[k]) {
-                    const uint32_t rm = rmax[cur.row[k]];
-                    if (mag16_nonfinite<DT>(rm)) status |= MOFQ_STATUS_NONFINITE_INPUT;
-                    kqmath::Sc<NC> sc;
-                    S s_c, s_g;
-#pragma unroll
-                    for (int j = 0; j < NC; ++j) {
-                        if (DT == MOFQ_F16) kqmath::scale_pair_fast(mag16_to_float<DT>(rm), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
-                        else scale_pair(mag16_to_float<DT>(rm), p.rq.q[j], sc.s[j], sc.inv[j], status);
-                    }
-                    s_c.begin(sc);
-                    if (GRP) {
-#pragma unroll
-                        for (int j = 0; j < NC; ++j) {
-                            if (DT == MOFQ_F16) kqmath::scale_pair_fast(mag16_to_float<DT>(cur.segmax[k]), p.rq.q[j], p.rq.rq[j], sc.s[j], sc.inv[j]);
-                            else scale_pair(mag16_to_float<DT>(cur.segmax[k]), p.rq.q[j], sc.s[j], sc.inv[j], status);
-                        }
-                        s_g.begin(sc);
-                    }
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const uint4 v = lds128(cur.a0[k] ^ (uint32_t)(j << 4));
-                        s_c.chunk(v);
-                        if (GRP) s_g.chunk(v);
-                    }
-                    double a_c[NC], a_g[NC];
-#pragma unroll
-                    for (int j = 0; j < NC; ++j) a_c[j] = a_g[j] = 0.0;
-                    s_c.end(a_c);
-                    if (GRP) {
-                        s_g.end(a_g);
-#pragma unroll
-                        for (int j = 0; j < NC; ++j) {
-                            dacc[j] += p.grp_first ? a_g[j] : a_c[j];
-                            dacc[NC + j] += p.grp_first ? a_c[j] : a_g[j];
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < NC; ++j) dacc[j] += a_c[j];
-                    }
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[s2]);
-            if (++s2 == p.stages) s2 = 0;
-            cur = nxt;
-        }
-    }
-    // the previous launch on the stream has finished with the header and the partial sums once this returns
-    // (a no-op when this launch was not started early)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    block_finish<NA>(dacc, status, hdr, partials, fin, red);
-}
-
 // ---- per-tensor scale: abs-max kernel, then a streaming scoring kernel -----------------------------------
 template <int DT>
 __global__ void __launch_bounds__(256)
@@ -1304,95 +1096,6 @@ int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st)
     MOFQ_CUDA_OK(cudaGetLastError());
     return MOFQ_OK;
 }
-
-namespace {
-
-int launch_score_rows_stream(const ScoreJob &job, bool has_grp, cudaStream_t st)
-{
-    const mofq_tensor &x = job.x;
-    const int spr = (int)(x.cols / 128);
-    const int row_bytes = (int)x.cols * 2;
-    // tile shape: as many whole rows as fit in 36 KB, at most two 128-element segments per consumer thread,
-    // consumers a multiple of 32
-    auto consumers_for = [&](int r, int max_rounds, int *rounds_out) {
-        const int nseg = r * spr;
-        for (int rounds = 1; rounds <= max_rounds; ++rounds) {
-            const int t = 32 * ((nseg + 32 * rounds - 1) / (32 * rounds));
-            if (t <= kRsMaxConsumers) {
-                *rounds_out = rounds;
-                return t;
-            }
-        }
-        return 0;
-    };
-    int best_r = 1, best_t = 0, best_rounds = 1;
-    while (best_r < kRsMaxRows && (long long)(best_r + 1) <= x.rows && (best_r + 1) * row_bytes <= 36864) ++best_r;
-    for (; best_r >= 1; --best_r)
-        if ((best_t = consumers_for(best_r, 2, &best_rounds)) != 0) break;
-    if (best_t && has_grp) {
-        // With two scale sets per element the lanes of a partly filled last warp cost the most: take a taller tile
-        // (two stages of up to 52 KB still leave two blocks per SM) when it fills the warps clearly better
-        // (6656-element rows: 104 of 128 lanes with two rows, 208 of 224 with four).
-        double util = (double)(best_r * spr) / (double)(best_t * best_rounds);
-        for (int r = best_r + 1; r <= kRsMaxRows && r <= x.rows && r * row_bytes <= 53248; ++r) {
-            int rounds = 1;
-            const int t = consumers_for(r, 1, &rounds);
-            if (t && (double)(r * spr) / t > util + 0.1) {
-                util = (double)(r * spr) / t;
-                best_r = r;
-                best_t = t;
-            }
-        }
-    }
-    if (!best_t) return MOFQ_ERR_UNSUPPORTED;
-    RsParams p{};
-    p.x = static_cast<const uint16_t *>(x.data);
-    p.rows = x.rows;
-    p.ld = x.ld;
-    p.cols = (int)x.cols;
-    p.rows_per_tile = best_r;
-    p.segs_per_row = spr;
-    p.consumers = best_t;
-    p.stage_bytes = (best_r * row_bytes + 1023) & ~1023;
-    p.stages = 3 * p.stage_bytes + 2048 <= 113 * 1024 ? 3 : 2;   // keep two blocks per SM
-    // With two scale sets per element more resident warps hide more than a third stage does: two stages when that
-    // fits four blocks per SM (measured, 3 -> 2 stages: 6656-element rows 138.7 -> 129.7 us on 17920 rows,
-    // 11008-element rows 65.4 -> 55.0 us on 4096 rows).  The taller tiles above only fit with two anyway.
-    if (has_grp && 2 * p.stage_bytes + 2048 <= 56 * 1024) p.stages = 2;
-    p.grp_first = (job.gran == MOFQ_PER_GROUP) ? 1 : 0;
-    p.rq = job_rowq(job);
-    p.n_tiles = (x.rows + best_r - 1) / best_r;
-    const size_t smem = (size_t)p.stages * p.stage_bytes + 1024;
-    const int threads = best_t + 32;
-    const int k0 = job.cs.n_fp > 0 ? fp_kind_of(job.fp_formats[0]) : -1, k1 = job.cs.n_fp > 1 ? fp_kind_of(job.fp_formats[1]) : -1;
-    auto launch = [&](auto kernel) {
-        if (int rc = set_smem(kernel, smem)) return rc;
-        const int occ = std::max(1, blocks_per_sm((const void *)kernel, threads, smem));
-        long long grid = std::min<long long>(p.n_tiles, std::min<long long>((long long)sm_count() * occ, kMaxSlots));
-        p.tiles_per_cta = (p.n_tiles + grid - 1) / grid;
-        grid = (p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
-        // After another scoring launch of the same call this one may start before that one has drained (see the
-        // kernel's griddepcontrol pair); after anything else on the stream it starts in stream order as usual.
-        cudaLaunchConfig_t lc{};
-        lc.gridDim = dim3((unsigned)grid);
-        lc.blockDim = dim3((unsigned)threads);
-        lc.dynamicSmemBytes = smem;
-        lc.stream = st;
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[0].val.programmaticStreamSerializationAllowed = 1;
-        lc.attrs = at;
-        lc.numAttrs = job.overlap_prev ? 1 : 0;
-        MOFQ_CUDA_OK(cudaLaunchKernelEx(&lc, kernel, p, job.hdr, job.partials, job.fin));
-        return MOFQ_OK;
-    };
-    return dispatch_kinds(x.dtype, job.cs.n_int, k0, k1, [&](auto DT, auto NI, auto K0, auto K1) {
-        if (has_grp) return launch(kq_score_rows_stream<DT(), NI(), K0(), K1(), true>);
-        return launch(kq_score_rows_stream<DT(), NI(), K0(), K1(), false>);
-    });
-}
-
-}  // namespace
 
 int launch_score(const ScoreJob &job, cudaStream_t st)
 {

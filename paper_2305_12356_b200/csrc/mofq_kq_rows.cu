@@ -43,7 +43,7 @@ constexpr int kRmThreads = (kRmConsumerWarps + kRmScoutWarps + 1) * 32;    // + 
 constexpr int kRmTileCap = 70 * 1024;                      // most bytes of one tile (two rows of 17920 fp16)
 constexpr int kRmMaxSeg = kRmTileCap / 256;                // segments (= most rows) of one tile
 constexpr int kRmSlots = 6;                                // tiles in flight: barrier sets and per-tile tables
-constexpr int kRmRingBytes = 212 * 1024;                   // shared-memory ring: 3 tiles of 70 KB, 5 of 40 KB, 6 of <= 35 KB
+constexpr int kRmRingBytes = 3 * kRmTileCap;               // shared-memory ring: 3 tiles of 70 KB, 5 of 40 KB, 6 of <= 35 KB
 constexpr int kRmSlotMeta = 2 * kRmMaxSeg * 4;             // per slot: abs-max pattern of every segment and of every row
 constexpr int kRmSmemBytes = kRmRingBytes + kRmSlots * kRmSlotMeta + 1024;   // + slack to align the ring
 
@@ -125,6 +125,7 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
     __shared__ RmTileInfo tinfo[kRmSlots];
     __shared__ int err;
     __shared__ int is_last;
+    __shared__ double red[kRmConsumerWarps][kMaxAcc];   // single tensor: the consumer warps' sums, then the last CTA's totals
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (smem_u32(smem) + 1023u) & ~1023u;
     unsigned char *const smem_al = smem + (smem_base - smem_u32(smem));
@@ -281,9 +282,14 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
 #pragma unroll
                 for (int o = 16; o; o >>= 1) dacc[j] += __shfl_xor_sync(0xffffffffu, dacc[j], o);
             if (lane == 0) {
-                const long long slot = L.slot_off + (long long)((int)blockIdx.x - L.first_cta) * kRmConsumerWarps + warp;
+                if (p.hdr) {      // single tensor: the CTA adds its warps' sums itself (below) and deposits one slot
 #pragma unroll
-                for (int j = 0; j < NA; ++j) p.partials[slot * kMaxAcc + j] = dacc[j];
+                    for (int j = 0; j < NA; ++j) red[warp][j] = dacc[j];
+                } else {
+                    const long long slot = L.slot_off + (long long)((int)blockIdx.x - L.first_cta) * kRmConsumerWarps + warp;
+#pragma unroll
+                    for (int j = 0; j < NA; ++j) p.partials[slot * kMaxAcc + j] = dacc[j];
+                }
             }
             status = __reduce_or_sync(0xffffffffu, status);
             if (status && lane == 0) atomicOr(&p.status[p.layers ? cur_layer : 0], status);
@@ -361,7 +367,15 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
     }
     if (!p.hdr) return;
 
-    // ---------------- single tensor: the last CTA to finish adds the slots in order and writes the outputs ----------------
+    // ---------------- single tensor: each CTA deposits the sum of its warps; the last CTA to finish adds the CTAs' sums in
+    // order and writes the outputs ----------------
+    if (n_it == 0 && warp < kRmConsumerWarps && lane < NA) red[warp][lane] = 0.0;   // (cannot happen: every CTA has a tile)
+    __syncthreads();
+    if (tid < NA) {
+        double t = 0.0;
+        for (int w = 0; w < kRmConsumerWarps; ++w) t += red[w][tid];
+        p.partials[(size_t)blockIdx.x * kMaxAcc + tid] = t;
+    }
     __syncthreads();
     if (tid == 0) {
         __threadfence();
@@ -374,10 +388,9 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
     double tot[NA];
 #pragma unroll
     for (int j = 0; j < NA; ++j) tot[j] = 0.0;
-    const int n_slots = (int)gridDim.x * kRmConsumerWarps;
-    for (int slot = lane; slot < n_slots; slot += 32)
+    for (int c = lane; c < (int)gridDim.x; c += 32)     // lane l: CTAs l, l + 32, ... in that order
 #pragma unroll
-        for (int j = 0; j < NA; ++j) tot[j] += __ldcg(&p.partials[(size_t)slot * kMaxAcc + j]);
+        for (int j = 0; j < NA; ++j) tot[j] += __ldcg(&p.partials[(size_t)c * kMaxAcc + j]);
 #pragma unroll
     for (int j = 0; j < NA; ++j)
 #pragma unroll

@@ -69,6 +69,40 @@ def test_llama33b_channel_and_group_full_size_layers(orc, dev):
     torch.cuda.empty_cache()
 
 
+def test_mixed_winners_at_full_layer_shapes(orc, dev):
+    """Decisions that can go either way, at the workloads' layer shapes: flat-distributed layers (the INT grid wins)
+    between heavy-tailed ones (the FP grid wins), scored in one call under per-channel and group-128 scales."""
+    g = torch.Generator().manual_seed(91)
+    layers = []
+    for li, (o, i, kind) in enumerate([(4096, 4096, "flat"), (11008, 4096, "student_t"), (4096, 11008, "flat"), (6656, 6656, "laplace")]):
+        if kind == "flat":
+            w = ((torch.rand((o, i), generator=g) - 0.5) * 0.1).to(torch.float16).to(dev)
+        else:
+            w = inputs.device_weight(torch.empty((o, i), dtype=torch.float16, device=dev), kind, 92, li)
+        layers.append(w)
+    names = ["INT4", "FP4_E2M1"]
+    cands = [orc.INT4, orc.FP4_E2M1]
+    cfg = mofq.make_config(4, names, w_gran="channel", w_group=128, w_gran2="group")
+    recs = mofq.select_formats(layers, cfg)
+    only_group = mofq.select_formats(layers, mofq.make_config(4, names, w_gran="group", w_group=128))   # the multi-tensor kernel
+    winners = set()
+    for li, w in enumerate(layers):
+        wh = host(w)
+        for s, (gr, grp) in enumerate(((orc.PER_CHANNEL, 0), (orc.PER_GROUP, 128))):
+            want = [orc.tensor_mse(wh, f, gr, grp) for f in cands]
+            r = recs[2 * li + s]
+            assert r["status"] == 0
+            assert rel_err(r["errors"], want).max() < MSE_RTOL, (li, s, r, want)
+            assert r["chosen"] == orc.select(want), (li, s, r, want)
+            winners.add(r["chosen"])
+            if s == 1:
+                assert rel_err(only_group[li]["errors"], want).max() < MSE_RTOL
+                assert only_group[li]["chosen"] == r["chosen"]
+    assert winners == {0, 1}, "the fixture is meant to produce both winners"
+    del layers
+    torch.cuda.empty_cache()
+
+
 @pytest.mark.parametrize("name,layer_index", [("llama65b_w8a8_layer", 6), ("llama13b_w8a8_layer", 4)])
 def test_layer_output_full_size_one_hot_activations(orc, dev, name, layer_index):
     """X = T one-hot rows: Y[t,:] is column c_t of W, and (the value 1 being exact in every format) the quantised

@@ -52,6 +52,24 @@ def test_layer_output_error_matches_oracle(orc, dev, T, n_in, n_out, names, w_on
     assert rel_err(nsr.cpu().numpy(), want_nsr).max() < LAYER_RTOL, (nsr, want_nsr)
 
 
+@pytest.mark.parametrize("T,n_in,n_out", [(512, 1024, 8192), (256, 22016, 512)])
+def test_dense_outlier_activations_paired_tiles_and_full_depth(orc, dev, T, n_in, n_out):
+    """Dense calibration activations with outlier channels (the 65B-shaped workload's recipe) at sizes whose cost
+    model picks the two-CTA 256 x 256 tile (512 x 8192 outputs) and at the workload's deepest contraction
+    (22016 input features): every output is a long accumulation of real products, unlike the one-hot cases."""
+    a_args = dict(n_ch=8, ch_gain=80.0, row_frac=0.0, row_gain=1.0)
+    w, x = _layer(dev, T, n_in, n_out, seed=56, layer=3, a_args=a_args)
+    names = ["INT8", "FP8_E4M3"]
+    cfg = mofq.make_config(8, names, metric="layer_output", is_w_only=False, w_gran="channel", a_gran="tensor")
+    rec = mofq.select_formats([(w, x)], cfg)[0]
+    want_mse, want_nsr = _oracle(orc, w, x, names, False)
+    assert rec["status"] == 0
+    assert rel_err(rec["errors"], want_mse).max() < LAYER_RTOL, (rec, want_mse)
+    assert rel_err(rec["nsr"], want_nsr).max() < LAYER_RTOL, (rec, want_nsr)
+    assert rec["chosen"] == orc.select(want_mse)
+    assert rec["chosen"] == 1                       # activation outliers: the floating-point grid wins (Section 3.2)
+
+
 def test_wide_tile_variant(orc, dev):
     # 2 x 74 tiles of 128 x 256 fill 148 SMs in one wave, so the 256-wide tile is chosen; the right edge is ragged
     T, n_in, n_out = 256, 128, 18936

@@ -8,6 +8,7 @@ that pytest collects it last.
 """
 import ctypes as C
 
+import numpy as np
 import pytest
 import torch
 
@@ -52,6 +53,35 @@ def test_noalloc_matches_workspace_entry_point_on_two_calls_in_a_row():
     want3, _ = mofq.tensor_error(a, cands, "channel")
     torch.cuda.synchronize()
     assert int(s3.item()) == 0 and torch.allclose(o3, want3, rtol=MSE_RTOL, atol=0.0)
+
+
+def test_noalloc_matches_the_oracle_and_takes_the_large_tensor_route(orc):
+    """The numbers are checked against the CPU oracle directly (not only against the sibling entry point), and a dense
+    tensor of more than 32 Mi elements with group scales goes through the persistent multi-tensor kernel, whose work
+    table, partial sums and status words then all live inside the built-in scratch; a small call right after it
+    must not see what that left behind."""
+    dev = torch.device("cuda:0")
+    cands = ["INT4", "FP4_E2M1"]
+    fm = [orc.INT4, orc.FP4_E2M1]
+    small = _weights(dev, 96, 1152, "laplace", 44, 0)
+    big = _weights(dev, 8192, 8192, "student_t", 45, 1)      # 64 Mi elements = 128 MiB of fp16
+    o_big = torch.empty(2, dtype=torch.float32, device=dev)
+    o_small = torch.empty((2, 2), dtype=torch.float32, device=dev)
+    s_big = torch.full((1,), -1, dtype=torch.int32, device=dev)
+    s_small = torch.full((1,), -1, dtype=torch.int32, device=dev)
+    mofq.tensor_error_noalloc(big, cands, "group", group=128, mse_out=o_big, status_out=s_big)
+    mofq.tensor_error_noalloc(small, cands, "channel", gran2="group", group=128, mse_out=o_small, status_out=s_small)
+    torch.cuda.synchronize()
+    assert int(s_big.item()) == 0 and int(s_small.item()) == 0
+    rows = torch.arange(0, 8192, 37)                          # the oracle scores a row sample of the large tensor ...
+    sample = big[rows.to(dev)].contiguous()
+    got_sample, _ = mofq.tensor_error(sample, cands, "group", group=128)
+    want_sample = [orc.tensor_mse(sample.cpu(), f, orc.PER_GROUP, 128) for f in fm]
+    assert np.allclose(got_sample.cpu().numpy(), want_sample, rtol=MSE_RTOL, atol=0)
+    want_big, _ = mofq.tensor_error(big, cands, "group", group=128)      # ... and the whole of it must agree with the workspace path
+    assert torch.allclose(o_big, want_big, rtol=MSE_RTOL, atol=0.0)
+    want_small = [[orc.tensor_mse(small.cpu(), f, g, 128) for f in fm] for g in (orc.PER_CHANNEL, orc.PER_GROUP)]
+    assert np.allclose(o_small.cpu().numpy(), want_small, rtol=MSE_RTOL, atol=0)
 
 
 def test_noalloc_rejects_tensors_beyond_its_limit():
