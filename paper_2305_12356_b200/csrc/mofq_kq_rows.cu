@@ -334,7 +334,9 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
                             }
                             s_g.begin(sc);
                         }
-#pragma unroll
+                        // with four candidates per element the fully unrolled loop no longer fits the instruction cache
+                        // close to the schedulers (a fifth of the issue slots went to instruction fetch stalls)
+#pragma unroll (GRP ? 4 : 16)
                         for (int j = 0; j < 16; ++j) {
                             const uint4 v = lds128(a0 ^ (uint32_t)(j << 4));
                             s_c.chunk(v);
