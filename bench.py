@@ -38,7 +38,8 @@ WORKLOAD_ORDER = ["single_4096_w4_channel", "llama7b_w4_group128", "llama13b_w8a
 # DRAM bytes per element of the scoring kernels, from the ncu captures summarised in profiles/ (read + write bytes
 # over the elements of the captured case; traffic is proportional to the elements processed).  None: not captured
 # for the kernel as it stands.
-DRAM_BYTES_PER_ELEMENT = {"kq_score_mt": None, "kq_score_rows_mt": None}
+DRAM_BYTES_PER_ELEMENT = {"kq_score_mt": (809.68e6 + 3.94e6) / 404750336,          # 14 layers of the 7B-shaped model
+                          "kq_score_rows_mt": (2140.26e6 + 4.26e6) / 1070071808}  # 14 layers of the 33B-shaped model
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 L2_BYTES = 126e6
@@ -472,7 +473,7 @@ def main():
 
     import paper_2305_12356_b200 as mofq
     from paper_2305_12356_b200 import inputs
-    from paper_2305_12356_b200.sharded import max_over_ranks, partition_layers, select_formats_sharded
+    from paper_2305_12356_b200.sharded import layer_costs, max_over_ranks, partition_layers, select_formats_sharded
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -502,9 +503,8 @@ def main():
     if sharded:
         # ONE model, its layer list split over the ranks by cost (bytes of W for the tensor criterion, flops for the
         # layer-output criterion); no tensor data moves between GPUs, the records are gathered on the host
-        shapes_all = inputs.workload_layers(args.workload, args.blocks)
         wl0 = inputs.WORKLOADS[args.workload]
-        costs = [o * i * (wl0["tokens"] if wl0["metric"] == "layer_output" else 1) for _, o, i in shapes_all]
+        costs = layer_costs(inputs.workload_layers(args.workload, args.blocks), wl0["metric"], wl0["tokens"])
         subset = partition_layers(costs, world)[rank]
     w = Workload(args.workload, dev, 0 if sharded else rank, args.blocks, subset)
     barrier()

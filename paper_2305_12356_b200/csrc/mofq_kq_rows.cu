@@ -23,7 +23,9 @@
 
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 #include <type_traits>
+#include <utility>
 #include <vector>
 
 #include "kq_finish.cuh"
@@ -582,14 +584,33 @@ bool make_plan(const mofq_tensor *const *tensors, int n, RmPlan *plan)
     return true;
 }
 
+// The kernel always asks for the same amount of dynamic shared memory, so the opt-in is made once per (device, kernel)
+// and remembered: a single small tensor's call is short enough for the repeated attribute call to show.
+int smem_opt_in(const void *kernel)
+{
+    static std::mutex mu;
+    static std::vector<std::pair<int, const void *>> done;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MOFQ_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    for (const auto &d : done)
+        if (d.first == dev && d.second == kernel) return MOFQ_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRmSmemBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MOFQ_ERR_CUDA;
+    }
+    done.emplace_back(dev, kernel);
+    return MOFQ_OK;
+}
+
 template <typename K>
 int launch_kernel(K kernel, const RmPlan &plan, const RmParams &p, cudaStream_t st)
 {
     const size_t smem = kRmSmemBytes;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return MOFQ_ERR_CUDA;
-    }
+    if (int rc = smem_opt_in(reinterpret_cast<const void *>(kernel))) return rc;
     kernel<<<plan.grid, kRmThreads, smem, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
     return MOFQ_OK;

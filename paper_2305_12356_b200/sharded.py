@@ -24,6 +24,14 @@ def partition_layers(costs, world):
     return [sorted(p) for p in parts]
 
 
+def layer_costs(shapes, metric="tensor", tokens=0):
+    """Per-layer balancing cost for [(name, out_features, in_features)]: bytes of W under the tensor criterion (the
+    scoring kernels are bound by the read of W), multiply-adds of the layer under the layer-output criterion."""
+    if metric == "layer_output":
+        return [o * i * max(1, tokens) for _, o, i in shapes]
+    return [2 * o * i for _, o, i in shapes]
+
+
 def select_formats_sharded(costs, score_fn, group=None):
     """Score this rank's share of the layers and return the records of ALL layers, in layer order, on every rank.
 
