@@ -403,6 +403,19 @@ def measure(w, args, barrier, peaks, which, steps, warmup, flusher):
     return rec
 
 
+def emit_winners_ms(w, barrier):
+    """Algorithm 1's last step, for context (not part of the metric): every layer quantised to its winner, which the
+    kernels read on the device from the records the last selection step left."""
+    import torch
+    import paper_2305_12356_b200 as mofq
+    from paper_2305_12356_b200 import binding as B
+    bufs = B.EmitBuffers(w.prepared, w.cfg)
+    ms = time_loop(lambda: mofq.emit_selected(w.prepared, w.cfg, w.results, buffers=bufs), 2, 1, barrier)
+    assert int(bufs.ws[:4].view(torch.int32).item()) == 0
+    del bufs
+    return ms
+
+
 def e2e_pass(w, args, dev, barrier, world):
     """The same metric through mofq_select_formats_host: pinned host tensors, host->device copies and the read-back of
     the records inside the timed region.  Bounded to the workload's first layers (args.e2e_gb of fp16) so that the
@@ -552,6 +565,8 @@ def main():
                                              "frac": w.fp16_bytes / (burst_ms * 1e-3) / 1e9 / head["roofline"]["peak"],
                                              "note": "median of 5 steps launched alone after 50 ms idle (no power-cap throttling); context only"}
 
+    if rank == 0 and w.grans == ("group",) and not w.layer_metric and not w.streaming and w.fp16_bytes < 40e9:
+        head["emit_winners_ms"] = emit_winners_ms(w, barrier)
     e2e = None
     if not args.no_e2e:
         e2e = e2e_pass(w, args, dev, barrier, world)
@@ -570,13 +585,7 @@ def main():
             rec = measure(ow, args, barrier, peaks, which, steps, 3, flusher)
             rec["config_index"] = WORKLOAD_ORDER.index(name) + 1
             if ow.grans == ("group",) and not ow.layer_metric:
-                # Algorithm 1's last step, for context (not part of the metric): every layer quantised to its winner,
-                # read on the device from the records the last step left
-                from paper_2305_12356_b200 import binding as B
-                bufs = B.EmitBuffers(ow.prepared, ow.cfg)
-                rec["emit_winners_ms"] = time_loop(lambda: mofq.emit_selected(ow.prepared, ow.cfg, ow.results, buffers=bufs), 2, 1, barrier)
-                assert int(bufs.ws[:4].view(torch.int32).item()) == 0
-                del bufs
+                rec["emit_winners_ms"] = emit_winners_ms(ow, barrier)
             if ow.layer_metric and not args.no_e2e:
                 rec["e2e"] = e2e_pass(ow, args, dev, barrier, world)
             if ow.layer_metric and not args.no_cpu_baseline:
