@@ -27,7 +27,12 @@
  *     mofq_select_formats / mofq_emit_selected after the layers before the refused one.
  *     Conditions found on the device (non-finite input, a reciprocal scale that overflows
  *     binary32) are reported as MOFQ_STATUS_* bits in a device status word.
- *   - Input values must be finite.
+ *   - Input values must be finite.  Every fp16 tensor and any bf16 tensor of magnitude below 1e18 is
+ *     in range for every call.  Beyond that (bf16 only) the whole-model selection kernels and the
+ *     per-tensor-scale scoring still work, because they sum squared errors in units of the scale;
+ *     mofq_select_blocks, group scales on a single small or strided tensor and
+ *     mofq_tensor_error_scaled sum unscaled squares in binary32 and report +Inf there.  A reported
+ *     error must itself fit binary32.
  *   - Candidates: at most MOFQ_MAX_CAND entries per call, of which at most one INT format and two
  *     distinct FP formats (three distinct formats); a list may repeat a format.
  *   - What the arithmetic contract below binds: the code-writing calls (mofq_quantize_tensor,

@@ -13,6 +13,7 @@
 //         the exact product once instead of twice; the two can differ only where a*inv sits within
 //         one binary32 ulp of a tie, and at a tie both neighbours have the same error, so the
 //         squared-error sum agrees with the two-rounding definition far inside the 1e-5 tolerance.
+//         d = r - a*inv (one fused operation); the group's sum of d*d is multiplied by scale^2 once per group.
 //   FP  : t = RN32(a*inv); r = hardware convert of t to the 4/8-bit float (round-to-nearest-even,
 //         saturating) and back to f16; d = r - t with a mixed-precision subtract; the group's sum of d*d is
 //         multiplied by scale^2 once per group (the scale is fixed over a lane's group).

@@ -150,6 +150,33 @@ def test_tensor_error_matches_oracle(orc, dev, names, gran, group, dtype):
     assert int(st.item()) == 0
 
 
+@pytest.mark.parametrize("absmax", [1.6e20, 1e-16])
+@pytest.mark.parametrize("gran,group,gran2", [("channel", 128, "group"), ("channel", 0, None), ("tensor", 0, None)])
+def test_tensor_error_bf16_extreme_magnitudes(orc, dev, absmax, gran, group, gran2):
+    """bfloat16 tensors whose largest scales, squared, leave the binary32 range (abs-max 1.6e20: scale^2 up to 7e38) or sit
+    a few decades above its subnormals (abs-max 1e-16: ~3e-34): the FP candidates' sums are kept in units of the scale
+    and scaled back in double, so the errors (which still fit binary32) and the decisions must agree with the oracle
+    as for ordinary magnitudes.  (Covers the kernels behind whole-model selection and per-tensor activation scales;
+    the block-wise selection kernel sums unscaled squares in binary32 and is documented to need |x| < 1e18.)"""
+    w = _weights(dev, 64, 1152, seed=23, layer=4).float()
+    x = (w * (absmax / float(w.abs().max()))).to(torch.bfloat16)
+    names = ["INT4", "FP4_E2M1"]
+    got, st = mofq.tensor_error(x, names, gran, gran2=gran2, group=group)
+    want = _oracle_mse(orc, host(x), names, gran, group if gran == "group" else 0)
+    if gran2:
+        want = want + _oracle_mse(orc, host(x), names, gran2, group)
+    assert int(st.item()) == 0
+    got = got.cpu().numpy().reshape(-1)
+    assert np.all(np.isfinite(got)) and np.all(got > 0)
+    assert rel_err(got, want).max() < MSE_RTOL, (got, want)
+    cfg = mofq.make_config(4, names, w_gran=gran, w_group=group, w_gran2=gran2)
+    recs = mofq.select_formats([x, x], cfg)
+    n_sets = 2 if gran2 else 1
+    for k, r in enumerate(recs):
+        w = want[(k % n_sets) * 2:(k % n_sets) * 2 + 2]
+        assert r["status"] == 0 and r["chosen"] == orc.select(w)
+
+
 @pytest.mark.parametrize("kind,kw", [("gauss_outlier", {}), ("laplace", {}), ("student_t", {})])
 def test_tensor_error_two_granularities_from_one_read(orc, dev, kind, kw):
     x = _weights(dev, 150, 6656, kind=kind, seed=22, layer=4)                 # LLaMA-33B hidden width: 52 groups per row
