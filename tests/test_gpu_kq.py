@@ -399,6 +399,53 @@ def test_streamed_rows_shapes(orc, dev, rows, cols, ld):
     assert rel_err(got2.cpu().numpy().reshape(-1), want2).max() < MSE_RTOL
 
 
+@pytest.mark.parametrize("rows,cols,group", [(37, 1000, 8), (9, 1096, 8), (3, 40000, 64), (70, 1160, 0)])
+def test_row_fallback_kernel_for_rows_the_streamed_kernel_does_not_take(orc, dev, rows, cols, group):
+    """Row lengths that are not a multiple of 128 elements, rows longer than the largest tile, and group sizes other
+    than 128 beside per-channel scales go through the one-row-per-CTA kernel."""
+    x = _weights(dev, rows, cols, seed=47, layer=rows % 5)
+    names = ["INT4", "FP4_E2M1"]
+    got, st = mofq.tensor_error(x, names, "channel", gran2="group" if group else None, group=group)
+    want = _oracle_mse(orc, host(x), names, "channel", 0)
+    if group:
+        want = want + _oracle_mse(orc, host(x), names, "group", group)
+    assert int(st.item()) == 0
+    assert rel_err(got.cpu().numpy().reshape(-1), want).max() < MSE_RTOL, (got, want)
+    cfg = mofq.make_config(4, names, w_gran="channel", w_group=group, w_gran2="group" if group else None)
+    recs = mofq.select_formats([x, x], cfg)                                # a list that the persistent kernel refuses
+    assert [r["chosen"] for r in recs[:len(recs) // 2]] == [orc.select(want[k:k + 2]) for k in range(0, len(want), 2)]
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_streamed_rows_random_layer_lists(orc, dev, seed):
+    """One persistent launch over lists of layers of unrelated shapes (single rows, rows of one segment, rows close
+    to the longest tile, more layers than CTAs' worth of work, a change of the ring's division at every layer): each
+    layer's errors and choice must be what the oracle gives for that layer alone, under every candidate set."""
+    rng = np.random.default_rng(100 + seed)
+    col_choices = [128, 256, 384, 1024, 2176, 4096, 6656, 11008, 17920, 24576, 35840]
+    shapes = [(int(rng.integers(1, 40 if c > 8000 else 200)), int(c)) for c in rng.choice(col_choices, size=23)]
+    shapes += [(1, 128), (1, 35840), (513, 128)]
+    dtype = (torch.float16, torch.bfloat16)[seed % 2]
+    xs = [_weights(dev, r, c, kind=("student_t", "laplace", "gauss_outlier")[i % 3], seed=60 + seed, layer=i, dtype=dtype)
+          for i, (r, c) in enumerate(shapes)]
+    cases = [(4, ["INT4", "FP4_E2M1"], "channel", "group"), (4, ["FP4_E2M1", "INT4"], "group", "channel"),
+             (8, ["INT8", "FP8_E4M3", "FP8_E5M2"], "channel", None), (4, ["FP4_E2M1_IEEE", "INT4", "FP4_E2M1"], "channel", "group")]
+    for bits, names, g1, g2 in (cases[seed % 4], cases[(seed + 2) % 4]):
+        cfg = mofq.make_config(bits, names, w_gran=g1, w_group=128, w_gran2=g2)
+        recs = mofq.select_formats(xs, cfg)
+        again = mofq.select_formats(xs, cfg)
+        assert recs == again                                              # fixed summation order
+        n_sets = 2 if g2 else 1
+        for i, x in enumerate(xs):
+            for s, g in enumerate((g1, g2)[:n_sets]):
+                want = _oracle_mse(orc, host(x), names, g, 128 if g == "group" else 0)
+                r = recs[i * n_sets + s]
+                assert r["status"] == 0
+                assert rel_err(r["errors"], want).max() < MSE_RTOL, (shapes[i], g, r, want)
+                if min(abs(a - b) for k, a in enumerate(want) for b in want[k + 1:]) > 1e-4 * max(want):
+                    assert r["chosen"] == orc.select(want), (shapes[i], g, r, want)
+
+
 def test_streamed_rows_layers_of_one_call_overlap_safely(orc, dev):
     """Within one selection call the streamed-row kernel lets the next layer's launch start before the current one has
     drained; the header and the partial sums they share are only touched after the earlier launch has completed.
