@@ -385,7 +385,7 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
         if (cfg->metric == MOFQ_TENSOR_MSE)
             rc = score_layer_tensor(layers[i].W, cfg, cs, perm, nc, fp_formats, results_out + (size_t)i * n_sets, nullptr, workspace, st);
         else
-            rc = layer_metric_run(layers[i], cfg, results_out + i, nullptr, nullptr, workspace, workspace_bytes, st);
+            rc = layer_metric_run(layers[i], cfg, results_out + i, nullptr, nullptr, workspace, workspace_bytes, st, i > 0);
         if (rc) return rc;
     }
     return MOFQ_OK;

@@ -4,9 +4,42 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "mofq.h"
 
 namespace mofq {
+
+// ---- chained launches ------------------------------------------------------------------------------------
+// The kernels of one library call that follow one another on the stream are launched with programmatic stream
+// serialisation: the next kernel's blocks may be scheduled and run their prologue while the previous kernel drains.
+// Every such kernel calls chain_enter() before its first global-memory access: it returns once the previous kernel
+// has completed and its writes are visible, so the order of the data is the plain stream order; what is saved is the
+// launch gap between short kernels.  Without the launch attribute both instructions do nothing.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_enter()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+}
+#endif
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool chained,
+                                  Args &&...args)
+{
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at;
+    lc.numAttrs = chained ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, kernel, std::forward<Args>(args)...);
+}
 
 // ---- format description used by the kernels ------------------------------------------------------
 // FP grid with E exponent bits, M mantissa bits, bias 2^(E-1)-1 (Section 2; Table 3 for E2M1):
@@ -121,7 +154,7 @@ struct EmitSel {
 
 // kernels' host launchers (mofq_kq.cu)
 int launch_score(const ScoreJob &job, cudaStream_t st);
-int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st);
+int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st, bool chained = false /* follows a kernel of the same call */);
 int launch_absmax_update(const mofq_tensor &x, float *absmax_inout, cudaStream_t st);
 int launch_score_supplied(const ScoreJob &job, const float *scales, cudaStream_t st);
 // one winner per scale block; job.fin.mse_out receives n_cand + 1 floats (candidates, then the mixture)
@@ -131,17 +164,21 @@ int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, con
                 WsHeader *hdr, cudaStream_t st, int format_id = -1 /* mofq_format of f: enables the fused code kernel */,
                 const EmitSel *sel = nullptr /* format chosen on the device; f then only fixes the code width */,
                 bool overlap_prev = false /* the previous launch on st is the previous layer's emission of the same call */);
+// x16_out / alpha_out (bf16 tensors only, nullable): also write the tensor as binary16, scaled by the power of two that
+// puts its abs-max in [2^13, 2^14) (exact unless a value is more than 2^27 times smaller than the abs-max), and 1 / that power
 int launch_emit_codes_uniform(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
-                              WsHeader *hdr, cudaStream_t st);
+                              WsHeader *hdr, cudaStream_t st, uint16_t *x16_out = nullptr, float *alpha_out = nullptr,
+                              bool chained = false);
 int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
-                           WsHeader *hdr, cudaStream_t st);
+                           WsHeader *hdr, cudaStream_t st, bool chained = false);
 
 // layer-output metric (mofq_layer.cu): extra workspace beyond the scoring workspace, and one layer's run.
 // Exactly one of `res` (selection record) or `mse_out`/`nsr_out` (raw errors, caller's order) is given.
 size_t layer_metric_ws_bytes(const mofq_layer *layers, int n_layers, const mofq_config *cfg);
 // the argument combinations layer_metric_run refuses (host-side checks only; nothing is enqueued)
 int layer_metric_check(const mofq_layer &L, const mofq_config *cfg);
+// after_own: the previous launch on st is the last kernel of the previous layer of the same call
 int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *res, float *mse_out, float *nsr_out,
-                     void *workspace, size_t workspace_bytes, cudaStream_t st);
+                     void *workspace, size_t workspace_bytes, cudaStream_t st, bool after_own = false);
 
 }  // namespace mofq

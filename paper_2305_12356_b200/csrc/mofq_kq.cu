@@ -357,6 +357,7 @@ template <int DT>
 __global__ void __launch_bounds__(256)
 kq_absmax(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, WsHeader *hdr)
 {
+    chain_enter();
     uint32_t m = 0;
     const long long total = rows * chunks_per_row;
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -863,12 +864,15 @@ struct EmitSet {
     float Q[3];
     unsigned char *codes[3];
     float *scales[3];
+    uint16_t *x16;     // per-tensor variant, bf16 input: the tensor as binary16 times a power of two (nullable)
+    float *alpha;      // 1 / that power of two
 };
 
 template <int DT>
 __global__ void __launch_bounds__(kRowThreads)
 kq_emit_codes_rows(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, EmitSet es, WsHeader *hdr)
 {
+    chain_enter();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint32_t mred[34];
     __shared__ float inv_s[3];
@@ -912,9 +916,19 @@ template <int DT>
 __global__ void __launch_bounds__(256)
 kq_emit_codes_uniform(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, EmitSet es, WsHeader *hdr)
 {
+    chain_enter();
     int status = 0;
     const uint32_t m16 = *reinterpret_cast<volatile uint32_t *>(&hdr->absmax_bits);
     if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
+    // binary16 copy of a bfloat16 tensor for the reference product: scaled by the power of two that puts the abs-max in
+    // [2^13, 2^14), which keeps every value exact unless it is more than 2^27 times smaller than the abs-max
+    float mult = 1.0f;
+    if (DT == MOFQ_BF16 && es.x16) {
+        const int e = (int)(m16 >> 7) - 127;
+        const int pw = m16 ? 13 - e : 0;
+        mult = exp2f((float)max(min(pw, 126), -126));
+        if (blockIdx.x == 0 && threadIdx.x == 0) *es.alpha = exp2f((float)-max(min(pw, 126), -126));
+    }
     float inv[3];
     for (int f = 0; f < es.n; ++f) {
         float s;
@@ -926,6 +940,16 @@ kq_emit_codes_uniform(const uint16_t *__restrict__ x, long long rows, int chunks
         const long long r = rows == 1 ? 0 : i / chunks_per_row;
         const int c = (int)(i - r * chunks_per_row);
         const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c);
+        if (DT == MOFQ_BF16 && es.x16) {
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float lo = __uint_as_float(w[k] << 16) * mult, hi = __uint_as_float(w[k] & 0xFFFF0000u) * mult;
+                o[k] = (uint32_t)__half_as_ushort(__float2half_rn(lo)) | ((uint32_t)__half_as_ushort(__float2half_rn(hi)) << 16);
+            }
+            reinterpret_cast<uint4 *>(es.x16)[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
         for (int f = 0; f < es.n; ++f) {
             const int fmt = es.format[f];
             const bool four = fmt == MOFQ_INT4 || fmt == MOFQ_FP4_E2M1 || fmt == MOFQ_FP4_E2M1_IEEE;
@@ -1083,17 +1107,16 @@ int launch_select_blocks(const ScoreJob &job, uint8_t *choice, float *block_sse,
     });
 }
 
-int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st)
+int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st, bool chained)
 {
     if (x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
     const long long total = x.rows * (x.cols / 8);
     const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
     if (x.dtype == MOFQ_F16)
-        kq_absmax<0><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, hdr);
+        MOFQ_CUDA_OK(launch_chained(kq_absmax<0>, dim3(grid), dim3(256), 0, st, chained, xp, (long long)x.rows, (int)(x.cols / 8), (long long)x.ld, hdr));
     else
-        kq_absmax<1><<<grid, 256, 0, st>>>(xp, x.rows, (int)(x.cols / 8), x.ld, hdr);
-    MOFQ_CUDA_OK(cudaGetLastError());
+        MOFQ_CUDA_OK(launch_chained(kq_absmax<1>, dim3(grid), dim3(256), 0, st, chained, xp, (long long)x.rows, (int)(x.cols / 8), (long long)x.ld, hdr));
     return MOFQ_OK;
 }
 
@@ -1159,11 +1182,14 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
 
 // Per-tensor scale from the abs-max already stored in hdr->absmax_bits (launch_absmax); codes of n formats from one read.
 int launch_emit_codes_uniform(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
-                              WsHeader *hdr, cudaStream_t st)
+                              WsHeader *hdr, cudaStream_t st, uint16_t *x16_out, float *alpha_out, bool chained)
 {
     if (n < 1 || n > 3 || x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+    if (x16_out && (x.dtype != MOFQ_BF16 || !alpha_out)) return MOFQ_ERR_INVALID_ARG;
     EmitSet es{};
     es.n = n;
+    es.x16 = x16_out;
+    es.alpha = alpha_out;
     for (int i = 0; i < n; ++i) {
         FmtDesc d;
         if (!describe_format(formats[i], &d)) return MOFQ_ERR_INVALID_ARG;
@@ -1180,16 +1206,15 @@ int launch_emit_codes_uniform(const mofq_tensor &x, int n, const int *formats, v
     const long long rows = flat ? 1 : x.rows;
     const int cpr = flat ? (int)total : (int)(x.cols / 8);
     if (x.dtype == MOFQ_F16)
-        kq_emit_codes_uniform<0><<<grid, 256, 0, st>>>(xp, rows, cpr, x.ld, es, hdr);
+        MOFQ_CUDA_OK(launch_chained(kq_emit_codes_uniform<0>, dim3(grid), dim3(256), 0, st, chained, xp, rows, cpr, (long long)x.ld, es, hdr));
     else
-        kq_emit_codes_uniform<1><<<grid, 256, 0, st>>>(xp, rows, cpr, x.ld, es, hdr);
-    MOFQ_CUDA_OK(cudaGetLastError());
+        MOFQ_CUDA_OK(launch_chained(kq_emit_codes_uniform<1>, dim3(grid), dim3(256), 0, st, chained, xp, rows, cpr, (long long)x.ld, es, hdr));
     return MOFQ_OK;
 }
 
 // Per-channel abs-max scales; codes (and scales) of n formats from one read.  formats[i] is a mofq_format.
 int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
-                           WsHeader *hdr, cudaStream_t st)
+                           WsHeader *hdr, cudaStream_t st, bool chained)
 {
     if (n < 1 || n > 3 || x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
     const size_t smem = (size_t)x.cols * 2;
@@ -1209,8 +1234,7 @@ int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void
         if (int rc = set_smem(kernel, smem)) return rc;
         const int occ = std::max(1, blocks_per_sm((const void *)kernel, kRowThreads, smem));
         const int grid = (int)std::min<long long>(x.rows, (long long)sm_count() * occ);
-        kernel<<<grid, kRowThreads, smem, st>>>(xp, x.rows, (int)x.cols, x.ld, es, hdr);
-        MOFQ_CUDA_OK(cudaGetLastError());
+        MOFQ_CUDA_OK(launch_chained(kernel, dim3(grid), dim3(kRowThreads), smem, st, chained, xp, (long long)x.rows, (int)x.cols, (long long)x.ld, es, hdr));
         return MOFQ_OK;
     };
     return x.dtype == MOFQ_F16 ? launch(kq_emit_codes_rows<0>) : launch(kq_emit_codes_rows<1>);

@@ -269,6 +269,7 @@ gemm_err_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ C
     else __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&tmem_base_slot);
+    chain_enter();   // barriers, tensor memory and descriptors are set up while the previous kernel of the call drains
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -542,6 +543,7 @@ gemm_err_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ C
 __global__ void __launch_bounds__(256)
 x_bf16_to_f16(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, const WsHeader *hdr, uint16_t *out, float *alpha_out)
 {
+    chain_enter();
     const uint32_t m16 = hdr->absmax_bits;
     const int e = (int)(m16 >> 7) - 127;  // bf16 exponent of the abs-max (0 -> treated as tiny)
     const int pw = m16 ? 13 - e : 0;
@@ -564,7 +566,11 @@ x_bf16_to_f16(const uint16_t *__restrict__ x, long long rows, int cols, long lon
     }
 }
 
-__global__ void set_scalar(float *p, float v) { *p = v; }
+__global__ void set_scalar(float *p, float v)
+{
+    chain_enter();
+    *p = v;
+}
 
 struct LayerFinalize {
     const double *partials;  // [(1 + n_cand)][stride]
@@ -574,11 +580,14 @@ struct LayerFinalize {
     mofq_result *res;
     float *mse_out, *nsr_out;
     int32_t *status;         // device status word: cleared after it is read when a record is written
+    uint32_t *absmax_bits;   // the header's activation abs-max: left zero for the next layer of the call
 };
 
 __global__ void __launch_bounds__(32)
 layer_finalize(const LayerFinalize f)
 {
+    chain_enter();
+    if (threadIdx.x == 0) *f.absmax_bits = 0;
     double tot[1 + MOFQ_MAX_CAND];
     for (int k = 0; k <= f.n_cand; ++k) {
         double s = 0.0;
@@ -683,7 +692,8 @@ constexpr int kOp8 = 100;
 // wave is shared instead of paid once per product.  n = 1 for the reference pass.
 int run_gemm_n(int n, const void *const *a, long long a_rows, const long long *a_ld, const void *const *b, long long b_rows,
                long long b_ld, long long K, const int *op, int mode, float *Y, const float *const *alpha,
-               const float *const *col_scale, double *const *partials, int32_t *status, int *grid_out, cudaStream_t st)
+               const float *const *col_scale, double *const *partials, int32_t *status, int *grid_out, cudaStream_t st,
+               bool chained = false)
 {
     if (n < 1 || n > kMaxProb) return MOFQ_ERR_INVALID_ARG;
     // tile shape: waves x relative tile cost.  Operand bytes per CTA and k-block: 32 KB for a 128x128 tile, 48 KB for
@@ -758,13 +768,15 @@ int run_gemm_n(int n, const void *const *a, long long a_rows, const long long *a
         lc.blockDim = dim3(kGemmThreads);
         lc.dynamicSmemBytes = smem;
         lc.stream = st;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)cg;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see chain_enter()
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         lc.attrs = attr;
-        lc.numAttrs = 1;
+        lc.numAttrs = chained ? 2 : 1;
         if (cudaLaunchKernelEx(&lc, kernel, maps, map_y, p) != cudaSuccess) {
             (void)cudaGetLastError();
             return MOFQ_ERR_CUDA;
@@ -780,9 +792,9 @@ int run_gemm_n(int n, const void *const *a, long long a_rows, const long long *a
 
 int run_gemm(const void *a, long long a_rows, long long a_ld, const void *b, long long b_rows, long long b_ld, long long K,
              int op, int mode, float *Y, const float *alpha, const float *col_scale, double *partials, int32_t *status,
-             int *grid_out, cudaStream_t st)
+             int *grid_out, cudaStream_t st, bool chained = false)
 {
-    return run_gemm_n(1, &a, a_rows, &a_ld, &b, b_rows, b_ld, K, &op, mode, Y, &alpha, &col_scale, &partials, status, grid_out, st);
+    return run_gemm_n(1, &a, a_rows, &a_ld, &b, b_rows, b_ld, K, &op, mode, Y, &alpha, &col_scale, &partials, status, grid_out, st, chained);
 }
 
 }  // namespace
@@ -813,7 +825,7 @@ int layer_metric_check(const mofq_layer &L, const mofq_config *cfg)
 }
 
 int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *res, float *mse_out, float *nsr_out,
-                     void *workspace, size_t workspace_bytes, cudaStream_t st)
+                     void *workspace, size_t workspace_bytes, cudaStream_t st, bool after_own)
 {
     const mofq_tensor &W = L.W, &X = L.X;
     if (int rc = layer_metric_check(L, cfg)) return rc;
@@ -837,20 +849,34 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
     long long xa_ld = X.ld;
     const bool native8 = !cfg->is_w_only && cfg->bit_width == 8 && (n_in % 16) == 0;
     const bool fused = native8 && cfg->n_candidates <= 3;
+    // The header's abs-max word is zero here: the entry points clear the header and every layer's finalize kernel leaves
+    // the word zero again.  Kernels of this layer after the first, and the first one after another layer of the same
+    // call, are chained launches (see chain_enter()).
+    bool chained = after_own;
     if (X.dtype != op_dtype || fused) {  // one abs-max of X serves the exact fp16 copy and the per-tensor activation scales
-        if (cudaMemsetAsync(&hdr->absmax_bits, 0, sizeof(uint32_t), st) != cudaSuccess) return MOFQ_ERR_CUDA;
-        if (int rc = launch_absmax(X, hdr, st)) return rc;
+        if (int rc = launch_absmax(X, hdr, st, chained)) return rc;
+        chained = true;
     }
+    const bool x16_with_codes = fused && X.dtype == MOFQ_BF16 && op_dtype == MOFQ_F16;   // written by the code-emission kernel below
     if (X.dtype != op_dtype) {  // bf16 activations with fp16 weights
-        const long long total = T * (n_in / 8);
-        const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
-        x_bf16_to_f16<<<grid, 256, 0, st>>>(static_cast<const uint16_t *>(X.data), T, (int)n_in, X.ld, hdr, x16, scal);
-        if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+        if (!x16_with_codes) {
+            const long long total = T * (n_in / 8);
+            const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
+            if (launch_chained(x_bf16_to_f16, dim3(grid), dim3(256), 0, st, chained, static_cast<const uint16_t *>(X.data), T, (int)n_in,
+                               (long long)X.ld, (const WsHeader *)hdr, x16, scal) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return MOFQ_ERR_CUDA;
+            }
+            chained = true;
+        }
         xa = x16;
         xa_ld = n_in;
     } else {
-        set_scalar<<<1, 1, 0, st>>>(scal, 1.0f);
-        if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+        if (launch_chained(set_scalar, dim3(1), dim3(1), 0, st, chained, scal, 1.0f) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MOFQ_ERR_CUDA;
+        }
+        chained = true;
     }
     // WA with 8-bit candidates: the codes themselves are the tensor-core operands (int8 / e4m3 / e5m2 kinds)
     // native path: the codes of every candidate from one read of W (one byte per element and format)
@@ -866,17 +892,22 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
             sptr[i] = sw + (size_t)i * sw_stride;
             fmts[i] = cfg->candidates[i];
         }
-        if (int rc = launch_emit_codes_rows(W, cfg->n_candidates, fmts, cptr, sptr, hdr, st)) return rc;
+        if (int rc = launch_emit_codes_rows(W, cfg->n_candidates, fmts, cptr, sptr, hdr, st, chained)) return rc;
+        chained = true;
         for (int i = 0; i < cfg->n_candidates; ++i) {  // activations: codes of every candidate, scales in scal[1 + i]
             cptr[i] = reinterpret_cast<unsigned char *>(cx) + (size_t)i * cx_stride;
             sptr[i] = scal + 1 + i;
         }
-        if (int rc = launch_emit_codes_uniform(X, cfg->n_candidates, fmts, cptr, sptr, hdr, st)) return rc;
+        // the same read of X also leaves its binary16 copy for the reference product
+        if (int rc = launch_emit_codes_uniform(X, cfg->n_candidates, fmts, cptr, sptr, hdr, st, x16_with_codes ? x16 : nullptr,
+                                               x16_with_codes ? scal : nullptr, chained))
+            return rc;
     }
     int grid_used = 0;
     int grids[1 + MOFQ_MAX_CAND] = {0};
-    if (int rc = run_gemm(xa, T, xa_ld, W.data, n_out, W.ld, n_in, op_dtype, 0, Y, scal, nullptr, partials, &hdr->status, &grid_used, st))
+    if (int rc = run_gemm(xa, T, xa_ld, W.data, n_out, W.ld, n_in, op_dtype, 0, Y, scal, nullptr, partials, &hdr->status, &grid_used, st, chained))
         return rc;
+    chained = true;
     grids[0] = grid_used;
     if (fused && cfg->n_candidates <= kMaxProb) {
         // every candidate's operands exist already: one launch carries all their products (Algorithm 1's loop over the
@@ -896,7 +927,7 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
             gpart[i] = partials + (size_t)(1 + i) * kMaxGemmCtas;
         }
         if (int rc = run_gemm_n(cfg->n_candidates, ga, T, gld, gb, n_out, n_in, n_in, gop, 1, Y, galpha, gcs, gpart, &hdr->status,
-                                &grid_used, st))
+                                &grid_used, st, true))
             return rc;
         for (int i = 0; i < cfg->n_candidates; ++i) grids[1 + i] = grid_used;
     } else {
@@ -941,8 +972,13 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
     f.mse_out = mse_out;
     f.nsr_out = nsr_out;
     f.status = &hdr->status;
-    layer_finalize<<<1, 32, 0, st>>>(f);
-    if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+    f.absmax_bits = &hdr->absmax_bits;
+    // (after the per-candidate loop of the general path the previous launch may be a memset-preceded kernel of the
+    // emission path: a chained launch behind a kernel that never signals simply starts when that kernel has finished)
+    if (launch_chained(layer_finalize, dim3(1), dim3(32), 0, st, true, f) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MOFQ_ERR_CUDA;
+    }
     return MOFQ_OK;
 }
 
