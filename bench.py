@@ -338,11 +338,12 @@ def kernel_facts(w):
     F = w.cfg.n_candidates
     if w.layer_metric:
         gemm = 2 if w.wl["bits"] == 8 else 1 + F          # 8-bit W+A: the candidates' products share one launch
-        return "gemm_err_kernel", n * gemm, n * (gemm + 5) + (2 * n if w.streaming else 0)
+        # per layer besides the products: activation abs-max, weight codes, activation codes (+ fp16 copy), finalize
+        return "gemm_err_kernel", n * gemm, n * (gemm + 4) + (2 * n if w.streaming else 0)
     if w.grans == ("group",):
         return "kq_score_mt", 1, 2 + (n + 63) // 64        # table uploads (64 layers each) + persistent kernel + finalize
     if n == 1:
-        return "kq_score_rows_mt", 1, 1                    # one launch: the last block applies Algorithm 1's comparison
+        return "kq_score_rows_mt", 1, 2                    # header clear + scoring launch (its last block applies Algorithm 1's comparison)
     return "kq_score_rows_mt", 1, 2 + (n + 31) // 32
 
 

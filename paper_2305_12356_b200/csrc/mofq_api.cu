@@ -115,8 +115,9 @@ int check_config(const mofq_config *cfg)
 }
 
 // tensor metric for one layer: enqueue the scoring of W and the record(s) for it
+// clear_header: the call has not cleared the workspace header yet
 int score_layer_tensor(const mofq_tensor &W, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
-                       const int *fp_formats, mofq_result *res, float *mse_out, void *ws, cudaStream_t st)
+                       const int *fp_formats, mofq_result *res, float *mse_out, void *ws, cudaStream_t st, bool clear_header = false)
 {
     if (int rc = check_tensor(&W)) return rc;
     if (int rc = check_gran(cfg->w_gran, cfg->w_group, W.cols)) return rc;
@@ -129,9 +130,11 @@ int score_layer_tensor(const mofq_tensor &W, const mofq_config *cfg, const CandS
     mofq_layer one{};
     one.W = W;
     if (cfg->metric == MOFQ_TENSOR_MSE && W.rows * W.cols >= (32LL << 20) && mt_applicable(&one, 1, cfg) &&
-        sizeof(WsHeader) + mt_ws_bytes(1) <= score_ws_bytes())
+        sizeof(WsHeader) + mt_ws_bytes(1) <= score_ws_bytes()) {
+        if (clear_header && cudaMemsetAsync(ws, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
         return mt_run(&one, 1, cfg, cs, perm, nc, fp_formats, res, static_cast<char *>(ws) + sizeof(WsHeader), st, mse_out,
                       res ? nullptr : &static_cast<WsHeader *>(ws)->status);   // a record carries its own status
+    }
     ScoreJob job{};
     job.x = W;
     job.cs = cs;
@@ -150,6 +153,7 @@ int score_layer_tensor(const mofq_tensor &W, const mofq_config *cfg, const CandS
     job.fin.nc = nc;
     std::memcpy(job.fin.perm, perm, sizeof(job.fin.perm));
     job.fin.inv_n = 1.0 / ((double)W.rows * (double)W.cols);
+    job.clear_header = clear_header;
     return launch_score(job, st);
 }
 
@@ -251,8 +255,7 @@ int mofq_tensor_error(const mofq_tensor *x, const int32_t *formats, int n, int g
     }
     if (int rc = check_ws(workspace, workspace_bytes, mofq_tensor_workspace_bytes(x))) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
-    return score_layer_tensor(*x, &cfg, cs, perm, nc, fp_formats, nullptr, mse_out, workspace, st);
+    return score_layer_tensor(*x, &cfg, cs, perm, nc, fp_formats, nullptr, mse_out, workspace, st, true);
 }
 
 int mofq_select_blocks(const mofq_tensor *x, const int32_t *formats, int n, int gran, int group, uint8_t *choice_out,
@@ -378,12 +381,12 @@ int mofq_select_formats(const mofq_layer *layers, int n_layers, const mofq_confi
     if (rows_mt_applicable(layers, n_layers, cfg))  // per-channel scales: one persistent launch over whole-row tiles
         return rows_mt_run(layers, n_layers, cfg, cs, perm, nc, fp_formats, results_out,
                            static_cast<char *>(workspace) + align256(score_ws_bytes()), st);
-    if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
+    if (cfg->metric != MOFQ_TENSOR_MSE && cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
     const int n_sets = cfg->w_gran2 != MOFQ_GRAN_NONE ? 2 : 1;
     for (int i = 0; i < n_layers; ++i) {  // Algorithm 1: for layer in model.layers_to_quant
         int rc;
-        if (cfg->metric == MOFQ_TENSOR_MSE)
-            rc = score_layer_tensor(layers[i].W, cfg, cs, perm, nc, fp_formats, results_out + (size_t)i * n_sets, nullptr, workspace, st);
+        if (cfg->metric == MOFQ_TENSOR_MSE)   // (the first layer's launch clears the workspace header)
+            rc = score_layer_tensor(layers[i].W, cfg, cs, perm, nc, fp_formats, results_out + (size_t)i * n_sets, nullptr, workspace, st, i == 0);
         else
             rc = layer_metric_run(layers[i], cfg, results_out + i, nullptr, nullptr, workspace, workspace_bytes, st, i > 0);
         if (rc) return rc;

@@ -22,6 +22,11 @@ __device__ __forceinline__ void chain_enter()
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
 }
+// The other form: a kernel entered with chain_enter_early() lets the launch chained behind it start at once; that
+// launch may read its inputs freely and calls chain_leave() before the first access to anything the earlier kernel
+// writes (used for the header clear in front of a single tensor's scoring launch).
+__device__ __forceinline__ void chain_enter_early() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void chain_leave() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 
 template <typename... KArgs, typename... Args>
@@ -107,6 +112,8 @@ struct ScoreJob {
     Finalize fin;
     WsHeader *hdr;
     double *partials;          // kMaxSlots * kMaxAcc doubles
+    bool clear_header;         // the call has not cleared *hdr yet: launch_score does it (for a single tensor on the
+                               // streamed-rows route with a kernel that the scoring launch overlaps, else with a memset)
 };
 
 inline size_t score_ws_bytes() { return sizeof(WsHeader) + sizeof(double) * kMaxSlots * kMaxAcc; }

@@ -1129,6 +1129,8 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
     const bool has_grp = job.gran == MOFQ_PER_GROUP || job.gran2 == MOFQ_PER_GROUP;
     const bool has_tensor = job.gran == MOFQ_PER_TENSOR || job.gran2 == MOFQ_PER_TENSOR;
     const int nsm = sm_count();
+    const bool rows_route = !has_tensor && has_ch && x.cols <= (1 << 20) && rows_single_applicable(job);
+    if (job.clear_header && !rows_route) MOFQ_CUDA_OK(cudaMemsetAsync(job.hdr, 0, sizeof(WsHeader), st));
 
     if (has_tensor) {
         if (job.gran2 != MOFQ_GRAN_NONE) return MOFQ_ERR_UNSUPPORTED;  // per-tensor cannot share a read
@@ -1157,7 +1159,7 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
 
     // row kernels: per-channel scales, alone or with group scales from the same read
     if (x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
-    if (rows_single_applicable(job)) return rows_single_run(job, st);
+    if (rows_route) return rows_single_run(job, st);
     const int chunks = (int)(x.cols / 8);
     const int gpr = has_grp ? (int)(x.cols / job.group) : 0;
     const size_t smem = (size_t)x.cols * 2 + (((size_t)chunks * 2 + 15) & ~(size_t)15) + (size_t)gpr * 8 * 3 + 16;

@@ -220,6 +220,7 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
                 const long long t0 = clock64();
                 while (!mbar_try_wait(&full_bar[k], 0) && !mbar_try_wait(&full_bar[k], 1) && clock64() - t0 < kWaitCycles) {}
             }
+            chain_leave();
             atomicOr(p.timeout, MOFQ_STATUS_TIMEOUT);
         }
     } else if (warp >= kRmConsumerWarps) {
@@ -266,7 +267,10 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
             __syncwarp();
             if (lane == 0) mbar_arrive(&row_bar[slot]);     // (release: the maxima above are visible to whoever waits)
         }
-        if (!ok && lane == 0) atomicOr(p.timeout, MOFQ_STATUS_TIMEOUT);
+        if (!ok && lane == 0) {
+            chain_leave();
+            atomicOr(p.timeout, MOFQ_STATUS_TIMEOUT);
+        }
     } else {
         // ---------------- consumer warps: pass 2 ----------------
         // The rounds of the CTA's tile sequence are numbered consecutively and warp w takes the rounds congruent to w:
@@ -294,7 +298,10 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
                 }
             }
             status = __reduce_or_sync(0xffffffffu, status);
-            if (status && lane == 0) atomicOr(&p.status[p.layers ? cur_layer : 0], status);
+            if (status && lane == 0) {
+                chain_leave();
+                atomicOr(&p.status[p.layers ? cur_layer : 0], status);
+            }
 #pragma unroll
             for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
             status = 0;
@@ -367,9 +374,15 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
             if (lane == 0) mbar_arrive(&empty_bar[slot]);
         }
         if (cur_layer >= 0) flush();
-        if (!ok && lane == 0) atomicOr(p.timeout, MOFQ_STATUS_TIMEOUT);   // a wait expired: the sums are incomplete
+        if (!ok && lane == 0) {   // a wait expired: the sums are incomplete
+            chain_leave();
+            atomicOr(p.timeout, MOFQ_STATUS_TIMEOUT);
+        }
     }
     if (!p.hdr) return;
+    // A single tensor's launch may have started beside the kernel that clears the workspace header (see
+    // kq_header_clear): the header is first touched below, or just above where a status bit is recorded.
+    chain_leave();
 
     // ---------------- single tensor: each CTA deposits the sum of its warps; the last CTA to finish adds the CTAs' sums in
     // order and writes the outputs ----------------
@@ -607,16 +620,27 @@ int smem_opt_in(const void *kernel)
 }
 
 template <typename K>
-int launch_kernel(K kernel, const RmPlan &plan, const RmParams &p, cudaStream_t st)
+int launch_kernel(K kernel, const RmPlan &plan, const RmParams &p, cudaStream_t st, bool chained)
 {
     const size_t smem = kRmSmemBytes;
     if (int rc = smem_opt_in(reinterpret_cast<const void *>(kernel))) return rc;
-    kernel<<<plan.grid, kRmThreads, smem, st>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+    if (launch_chained(kernel, dim3((unsigned)plan.grid), dim3(kRmThreads), smem, st, chained, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MOFQ_ERR_CUDA;
+    }
     return MOFQ_OK;
 }
 
-int launch_plan(const RmPlan &plan, RmParams &p, int dtype, const CandSet &cs, const int *fp_formats, bool has_grp, cudaStream_t st)
+// Clears a workspace header.  A single tensor's scoring launch is chained behind it and starts at once: that kernel
+// touches the header only after its chain_leave().
+__global__ void kq_header_clear(WsHeader *hdr)
+{
+    chain_enter_early();
+    reinterpret_cast<uint32_t *>(hdr)[threadIdx.x] = 0u;
+}
+
+int launch_plan(const RmPlan &plan, RmParams &p, int dtype, const CandSet &cs, const int *fp_formats, bool has_grp, cudaStream_t st,
+                bool chained = false)
 {
     p.n_layers = (int)plan.table.size();
     p.total_tiles = plan.total_tiles;
@@ -624,8 +648,8 @@ int launch_plan(const RmPlan &plan, RmParams &p, int dtype, const CandSet &cs, c
     p.rq = candset_rowq(cs);
     const int k0 = cs.n_fp > 0 ? fp_kind(fp_formats[0]) : -1, k1 = cs.n_fp > 1 ? fp_kind(fp_formats[1]) : -1;
     return dispatch_kinds(dtype, cs.n_int, k0, k1, [&](auto DT, auto NI, auto K0, auto K1) {
-        if (has_grp) return launch_kernel(kq_score_rows_mt<DT(), NI(), K0(), K1(), true>, plan, p, st);
-        return launch_kernel(kq_score_rows_mt<DT(), NI(), K0(), K1(), false>, plan, p, st);
+        if (has_grp) return launch_kernel(kq_score_rows_mt<DT(), NI(), K0(), K1(), true>, plan, p, st, chained);
+        return launch_kernel(kq_score_rows_mt<DT(), NI(), K0(), K1(), false>, plan, p, st, chained);
     });
 }
 
@@ -653,6 +677,10 @@ int rows_single_run(const ScoreJob &job, cudaStream_t st)
     const mofq_tensor *t = &job.x;
     if (!make_plan(&t, 1, &plan)) return MOFQ_ERR_UNSUPPORTED;
     if (plan.slots > kMaxSlots) return MOFQ_ERR_UNSUPPORTED;
+    if (job.clear_header) {
+        kq_header_clear<<<1, (unsigned)(sizeof(WsHeader) / sizeof(uint32_t)), 0, st>>>(job.hdr);
+        if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
+    }
     RmParams p{};
     p.layers = nullptr;
     p.one = plan.table[0];
@@ -663,7 +691,7 @@ int rows_single_run(const ScoreJob &job, cudaStream_t st)
     p.hdr = job.hdr;
     p.fin = job.fin;
     const bool has_grp = job.gran == MOFQ_PER_GROUP || job.gran2 == MOFQ_PER_GROUP;
-    return launch_plan(plan, p, job.x.dtype, job.cs, job.fp_formats, has_grp, st);
+    return launch_plan(plan, p, job.x.dtype, job.cs, job.fp_formats, has_grp, st, job.clear_header);
 }
 
 // A layer list under the tensor metric with per-channel scales (optionally group-128 scales as the other set) on
