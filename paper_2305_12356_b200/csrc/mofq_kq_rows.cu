@@ -405,9 +405,20 @@ kq_score_rows_mt(const __grid_constant__ RmParams p)
     double tot[NA];
 #pragma unroll
     for (int j = 0; j < NA; ++j) tot[j] = 0.0;
-    for (int c = lane; c < (int)gridDim.x; c += 32)     // lane l: CTAs l, l + 32, ... in that order
+    // lane l: CTAs l, l + 32, ... in that order; eight CTAs' slots are fetched before the first is added, so that the
+    // reduction costs one trip to the level-2 cache per 256 CTAs instead of one per 32
+    for (int c0 = lane; c0 < (int)gridDim.x; c0 += 32 * 8) {
+        double v[8][NA];
 #pragma unroll
-        for (int j = 0; j < NA; ++j) tot[j] += __ldcg(&p.partials[(size_t)c * kMaxAcc + j]);
+        for (int k = 0; k < 8; ++k)
+#pragma unroll
+            for (int j = 0; j < NA; ++j)
+                v[k][j] = c0 + 32 * k < (int)gridDim.x ? __ldcg(&p.partials[(size_t)(c0 + 32 * k) * kMaxAcc + j]) : 0.0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+#pragma unroll
+            for (int j = 0; j < NA; ++j) tot[j] += v[k][j];
+    }
 #pragma unroll
     for (int j = 0; j < NA; ++j)
 #pragma unroll
