@@ -15,7 +15,8 @@
  * precision; this file must be compiled with -ffp-contract=off and without -ffast-math.
  *
  * Pins (tests/test_oracle_*.py): Table 3 of the paper for the FP4 code->value map, enumeration
- * counts and library decodes for FP8, hand-made tie grids, closed-form uniform-noise MSE,
+ * counts and library decodes for FP8, hand-made tie grids, the scale pair against correctly
+ * rounded exact-rational quotients, closed-form uniform-noise MSE,
  * exact-rational brute force on tiny tensors, identity-activation and exact-integer special
  * cases for the layer output error; block-wise selection against row/group slices scored as
  * tensors of their own and a hand-worked two-row case.  No function in this file is "parity unpinned".

@@ -26,6 +26,10 @@ MUTATIONS = {
         "float Q = (float)f.fmt_max;",
         "float Q = (float)f.fmt_max + 1.0f;",
         "tests/test_oracle_quantize.py::test_scale_is_absmax_over_q"),
+    "inverse_scale_from_rounded_scale": (
+        "*inv = Q / absmax;",
+        "*inv = 1.0f / *scale;",
+        "tests/test_oracle_quantize.py::test_scale_pair_is_two_correctly_rounded_quotients"),
     "mse_divides_by_rows": (
         "sse / (double)(rows * cols)",
         "sse / (double)rows",

@@ -53,6 +53,44 @@ def test_scale_is_absmax_over_q(orc, name):
     assert qt["scales"].shape == (1,) and qt["scales"][0] == np.float32(1.5) / Q
 
 
+def _round_to_binary32(q):
+    """Correctly rounded (nearest, ties to even) binary32 of a positive exact rational in the normal range."""
+    e = 0
+    while q >= 2:
+        q /= 2
+        e += 1
+    while q < 1:
+        q *= 2
+        e -= 1
+    assert -126 <= e <= 127
+    m = q * (1 << 23)                       # 2^23 <= m < 2^24
+    n, rem = divmod(m.numerator, m.denominator)
+    twice = 2 * rem
+    if twice > m.denominator or (twice == m.denominator and (n & 1)):
+        n += 1
+    return np.float32(float(Fraction(n, 1 << 23) * Fraction(2) ** e))   # n <= 2^24: exact in binary64 and binary32
+
+
+@pytest.mark.parametrize("name", ALL_NAMES)
+def test_scale_pair_is_two_correctly_rounded_quotients(orc, name):
+    """scale = RN32(absmax / Q) and inv = RN32(Q / absmax), each rounded once from the exact quotient (exact rational
+    arithmetic here); in particular inv is NOT the reciprocal of the rounded scale."""
+    fmt = getattr(orc, name)
+    Q = Fraction(orc.format_max(fmt))
+    rng = np.random.default_rng(11)
+    bits = np.unique(np.concatenate([rng.integers(0x0001, 0x7C00, size=400), [0x0001, 0x03FF, 0x0400, 0x3C00, 0x7BFF]])).astype(np.uint16)
+    differs = 0
+    for b in bits:
+        a = np.array([b], dtype=np.uint16).view(np.float16)[0]
+        fa = Fraction(float(a))
+        scale, inv = orc.scale_from_absmax(fmt, float(a))
+        want_s, want_i = _round_to_binary32(fa / Q), _round_to_binary32(Q / fa)
+        assert np.float32(scale) == want_s and np.float32(inv) == want_i, (hex(int(b)), scale, inv, want_s, want_i)
+        differs += int(want_i != np.float32(1.0) / want_s)
+    assert differs > 0      # the sample tells the two definitions apart
+    assert orc.scale_from_absmax(fmt, 0.0) == (1.0, 1.0)
+
+
 @pytest.mark.parametrize("name", ALL_NAMES)
 def test_absmax_element_gets_top_code_and_no_reserved_codes(orc, name):
     fmt = getattr(orc, name)
