@@ -377,10 +377,9 @@ kq_absmax(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, lo
         const int c = (int)(i - r * chunks_per_row);
         m = absmax_chunk(__ldg(reinterpret_cast<const uint4 *>(x + r * ld) + c), m);
     }
-    uint32_t m16 = fold16(m);
-#pragma unroll
-    for (int o = 16; o; o >>= 1) m16 = max(m16, __shfl_xor_sync(0xffffffffu, m16, o));
-    if ((threadIdx.x & 31) == 0 && m16) atomicMax(&hdr->absmax_bits, m16);
+    __shared__ uint32_t mred[34];
+    const uint32_t m16 = block_max_u32(fold16(m), mred);   // one atomic per block: they all go to one address
+    if (threadIdx.x == 0 && m16) atomicMax(&hdr->absmax_bits, m16);
 }
 
 // The scale pairs are the same for every element, so the packed scorer runs in its scaled form; its binary32 chains
@@ -701,34 +700,32 @@ __device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
 // decoded once per kernel (it may have been picked on the device), not per element.
 enum { CLS_INT4 = 0, CLS_INT8 = 1, CLS_E2M1 = 2, CLS_E4M3 = 3, CLS_E5M2 = 4 };
 
-template <int DT, int CLS>
-__device__ __forceinline__ uint2 chunk_codes(const uint4 v, uint64_t inv2)
+// code(s) of one pair of elements (already widened to packed binary32); 8-bit classes: 16 bits, 4-bit classes: 8 bits
+template <int CLS>
+__device__ __forceinline__ uint32_t pair_code(uint64_t a2, uint64_t inv2)
 {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint32_t c[4];  // CLS with 8-bit codes: 16 bits per word; 4-bit codes: 8 bits per word
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint64_t a2 = kqmath::unpack2<DT>(w[i]);
-        float lo, hi;
-        if (CLS == CLS_INT4 || CLS == CLS_INT8) {
-            // t = RN32(x * inv) first (the code is decided on the rounded t), then the low mantissa bits of
-            // t + 1.5 * 2^23 are the two's-complement code
-            // (the add stays scalar: a packed multiply followed by a packed add came out as one fused operation,
-            // which rounds the exact product instead of t and breaks ties differently)
-            kqmath::upk(kqmath::mul2(a2, inv2), lo, hi);
-            lo = __fadd_rn(lo, kMagic);
-            hi = __fadd_rn(hi, kMagic);
-            uint32_t t = __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x0040);
-            if (CLS == CLS_INT4) {
-                t &= 0x0F0Fu;
-                t = (t | (t >> 4)) & 0xFFu;
-            }
-            c[i] = t;
-        } else {
-            kqmath::upk(kqmath::mul2(a2, inv2), lo, hi);
-            c[i] = CLS == CLS_E2M1 ? cvt_e2m1x2(lo, hi) : CLS == CLS_E4M3 ? cvt_e4m3x2(lo, hi) : cvt_e5m2x2(lo, hi);
+    float lo, hi;
+    kqmath::upk(kqmath::mul2(a2, inv2), lo, hi);   // t = RN32(x * inv) first: the code is decided on the rounded t
+    if (CLS == CLS_INT4 || CLS == CLS_INT8) {
+        // the low mantissa bits of t + 1.5 * 2^23 are the two's-complement code
+        // (the add stays scalar: a packed multiply followed by a packed add came out as one fused operation,
+        // which rounds the exact product instead of t and breaks ties differently)
+        lo = __fadd_rn(lo, kMagic);
+        hi = __fadd_rn(hi, kMagic);
+        uint32_t t = __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x0040);
+        if (CLS == CLS_INT4) {
+            t &= 0x0F0Fu;
+            t = (t | (t >> 4)) & 0xFFu;
         }
+        return t;
     }
+    return CLS == CLS_E2M1 ? cvt_e2m1x2(lo, hi) : CLS == CLS_E4M3 ? cvt_e4m3x2(lo, hi) : cvt_e5m2x2(lo, hi);
+}
+
+// four pair codes -> the chunk's codes, little-endian (8-bit classes: 64 bits, 4-bit classes: 32 bits in .x)
+template <int CLS>
+__device__ __forceinline__ uint2 pack_codes(const uint32_t (&c)[4])
+{
     uint2 o;
     if (CLS == CLS_INT4 || CLS == CLS_E2M1) {
         o.x = __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
@@ -738,6 +735,41 @@ __device__ __forceinline__ uint2 chunk_codes(const uint4 v, uint64_t inv2)
         o.y = __byte_perm(c[2], c[3], 0x5410);
     }
     return o;
+}
+
+template <int DT, int CLS>
+__device__ __forceinline__ uint2 chunk_codes(const uint4 v, uint64_t inv2)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t c[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] = pair_code<CLS>(kqmath::unpack2<DT>(w[i]), inv2);
+    return pack_codes<CLS>(c);
+}
+
+// the codes of up to three formats (classes C0, C1, C2; -1 = absent) from one widening of the chunk
+template <int DT, int C0, int C1, int C2>
+__device__ __forceinline__ void chunk_codes3(const uint4 v, const uint64_t (&inv2)[3], uint2 (&o)[3])
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t c0[4], c1[4], c2[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint64_t a2 = kqmath::unpack2<DT>(w[i]);
+        c0[i] = pair_code<C0>(a2, inv2[0]);
+        if (C1 >= 0) c1[i] = pair_code<(C1 >= 0 ? C1 : 0)>(a2, inv2[1]);
+        if (C2 >= 0) c2[i] = pair_code<(C2 >= 0 ? C2 : 0)>(a2, inv2[2]);
+    }
+    o[0] = pack_codes<C0>(c0);
+    if (C1 >= 0) o[1] = pack_codes<(C1 >= 0 ? C1 : 0)>(c1);
+    if (C2 >= 0) o[2] = pack_codes<(C2 >= 0 ? C2 : 0)>(c2);
+}
+
+template <int CLS>
+__device__ __forceinline__ void store_codes(unsigned char *base, size_t chunk, const uint2 o)
+{
+    if (CLS == CLS_INT4 || CLS == CLS_E2M1) reinterpret_cast<uint32_t *>(base)[chunk] = o.x;
+    else reinterpret_cast<uint2 *>(base)[chunk] = o;
 }
 
 template <int DT, int CLS>
@@ -842,37 +874,24 @@ kq_emit_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long lo
     if (status) atomicOr(&hdr->status, status);
 }
 
-// codes of 8 consecutive elements for one format, packed little-endian (8-bit: 64 bits, 4-bit: 32 bits)
-template <int DT>
-__device__ __forceinline__ uint64_t codes8(const uint4 v, int format, float inv)
-{
-    const uint64_t inv2 = kqmath::pk(inv, inv);
-    uint2 o;
-    switch (format) {  // uniform over the launch; the per-class code below is branch-free
-    case MOFQ_INT4: o = chunk_codes<DT, CLS_INT4>(v, inv2); break;
-    case MOFQ_INT8: o = chunk_codes<DT, CLS_INT8>(v, inv2); break;
-    case MOFQ_FP8_E4M3: o = chunk_codes<DT, CLS_E4M3>(v, inv2); break;
-    case MOFQ_FP8_E5M2: o = chunk_codes<DT, CLS_E5M2>(v, inv2); break;
-    default: o = chunk_codes<DT, CLS_E2M1>(v, inv2); break;  // both E2M1 variants: same spacing below the IEEE maximum 3
-    }
-    return (uint64_t)o.x | ((uint64_t)o.y << 32);
-}
-
 struct EmitSet {
     int n;
-    int format[3];
-    float Q[3];
+    float Q[3];                // formats in the kernel's class order C0, C1, C2
     unsigned char *codes[3];
     float *scales[3];
     uint16_t *x16;     // per-tensor variant, bf16 input: the tensor as binary16 times a power of two (nullable)
     float *alpha;      // 1 / that power of two
 };
 
-template <int DT>
+// Per-channel scales, codes of up to three formats (classes C0..C2 fixed at compile time, -1 = absent) from one staged
+// read of each row: one block per row at a time.
+template <int DT, int C0, int C1, int C2>
 __global__ void __launch_bounds__(kRowThreads)
 kq_emit_codes_rows(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, EmitSet es, WsHeader *hdr)
 {
     chain_enter();
+    constexpr int N = 1 + (C1 >= 0) + (C2 >= 0);
+    constexpr bool four = C0 == CLS_INT4 || C0 == CLS_E2M1;   // the classes of one launch share a code width
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint32_t mred[34];
     __shared__ float inv_s[3];
@@ -888,23 +907,25 @@ kq_emit_codes_rows(const uint16_t *__restrict__ x, long long rows, int cols, lon
         for (int q = threadIdx.x; q < chunks; q += kRowThreads) m = absmax_chunk(row4[q], m);
         const uint32_t m16 = block_max_u32(fold16(m), mred);
         if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
-        if ((int)threadIdx.x < es.n) {
-            float s, inv;
-            scale_pair(mag16_to_float<DT>(m16), es.Q[threadIdx.x], s, inv, status);
+        if ((int)threadIdx.x < N) {
+            float sc, inv;
+            scale_pair(mag16_to_float<DT>(m16), threadIdx.x == 0 ? es.Q[0] : threadIdx.x == 1 ? es.Q[1] : es.Q[2], sc, inv, status);
             inv_s[threadIdx.x] = inv;
-            if (es.scales[threadIdx.x]) es.scales[threadIdx.x][row] = s;
+            float *sp = threadIdx.x == 0 ? es.scales[0] : threadIdx.x == 1 ? es.scales[1] : es.scales[2];
+            if (sp) sp[row] = sc;
         }
         __syncthreads();
-        for (int f = 0; f < es.n; ++f) {
-            const float inv = inv_s[f];
-            const int fmt = es.format[f];
-            const bool four = fmt == MOFQ_INT4 || fmt == MOFQ_FP4_E2M1 || fmt == MOFQ_FP4_E2M1_IEEE;
-            unsigned char *out = es.codes[f] + (four ? ((size_t)row * cols >> 1) : (size_t)row * cols);
-            for (int q = threadIdx.x; q < chunks; q += kRowThreads) {
-                const uint64_t c = codes8<DT>(row4[q], fmt, inv);
-                if (four) reinterpret_cast<uint32_t *>(out)[q] = (uint32_t)c;
-                else reinterpret_cast<uint2 *>(out)[q] = make_uint2((uint32_t)c, (uint32_t)(c >> 32));
-            }
+        const uint64_t inv2[3] = {kqmath::pk(inv_s[0], inv_s[0]), kqmath::pk(inv_s[1], inv_s[1]), kqmath::pk(inv_s[2], inv_s[2])};
+        const size_t row_off = four ? ((size_t)row * cols >> 1) : (size_t)row * cols;
+        unsigned char *out0 = es.codes[0] + row_off, *out1 = N > 1 ? es.codes[1] + row_off : nullptr,
+                      *out2 = N > 2 ? es.codes[2] + row_off : nullptr;
+#pragma unroll 2
+        for (int q = threadIdx.x; q < chunks; q += kRowThreads) {
+            uint2 o[3];
+            chunk_codes3<DT, C0, C1, C2>(row4[q], inv2, o);
+            store_codes<C0>(out0, q, o[0]);
+            if (C1 >= 0) store_codes<(C1 >= 0 ? C1 : 0)>(out1, q, o[1]);
+            if (C2 >= 0) store_codes<(C2 >= 0 ? C2 : 0)>(out2, q, o[2]);
         }
         __syncthreads();
     }
@@ -912,11 +933,13 @@ kq_emit_codes_rows(const uint16_t *__restrict__ x, long long rows, int cols, lon
 }
 
 // per-tensor variant: the abs-max is already in the workspace header; codes of every requested format from one read
-template <int DT>
+template <int DT, int C0, int C1, int C2>
 __global__ void __launch_bounds__(256)
 kq_emit_codes_uniform(const uint16_t *__restrict__ x, long long rows, int chunks_per_row, long long ld, EmitSet es, WsHeader *hdr)
 {
     chain_enter();
+    constexpr int N = 1 + (C1 >= 0) + (C2 >= 0);
+    __shared__ float inv_s[3];
     int status = 0;
     const uint32_t m16 = *reinterpret_cast<volatile uint32_t *>(&hdr->absmax_bits);
     if (mag16_nonfinite<DT>(m16)) status |= MOFQ_STATUS_NONFINITE_INPUT;
@@ -929,12 +952,16 @@ kq_emit_codes_uniform(const uint16_t *__restrict__ x, long long rows, int chunks
         mult = exp2f((float)max(min(pw, 126), -126));
         if (blockIdx.x == 0 && threadIdx.x == 0) *es.alpha = exp2f((float)-max(min(pw, 126), -126));
     }
-    float inv[3];
-    for (int f = 0; f < es.n; ++f) {
-        float s;
-        scale_pair(mag16_to_float<DT>(m16), es.Q[f], s, inv[f], status);
-        if (blockIdx.x == 0 && threadIdx.x == 0 && es.scales[f]) es.scales[f][0] = s;
+    if ((int)threadIdx.x < N) {   // thread f forms format f's scale pair for the block
+        float sc, inv;
+        scale_pair(mag16_to_float<DT>(m16), threadIdx.x == 0 ? es.Q[0] : threadIdx.x == 1 ? es.Q[1] : es.Q[2], sc, inv, status);
+        inv_s[threadIdx.x] = inv;
+        float *sp = threadIdx.x == 0 ? es.scales[0] : threadIdx.x == 1 ? es.scales[1] : es.scales[2];
+        if (blockIdx.x == 0 && sp) sp[0] = sc;
     }
+    __syncthreads();
+    const uint64_t inv2[3] = {kqmath::pk(inv_s[0], inv_s[0]), kqmath::pk(inv_s[N > 1 ? 1 : 0], inv_s[N > 1 ? 1 : 0]),
+                              kqmath::pk(inv_s[N > 2 ? 2 : 0], inv_s[N > 2 ? 2 : 0])};
     const long long total = rows * chunks_per_row;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
         const long long r = rows == 1 ? 0 : i / chunks_per_row;
@@ -950,13 +977,11 @@ kq_emit_codes_uniform(const uint16_t *__restrict__ x, long long rows, int chunks
             }
             reinterpret_cast<uint4 *>(es.x16)[i] = make_uint4(o[0], o[1], o[2], o[3]);
         }
-        for (int f = 0; f < es.n; ++f) {
-            const int fmt = es.format[f];
-            const bool four = fmt == MOFQ_INT4 || fmt == MOFQ_FP4_E2M1 || fmt == MOFQ_FP4_E2M1_IEEE;
-            const uint64_t cd = codes8<DT>(v, fmt, inv[f]);
-            if (four) reinterpret_cast<uint32_t *>(es.codes[f])[i] = (uint32_t)cd;
-            else reinterpret_cast<uint2 *>(es.codes[f])[i] = make_uint2((uint32_t)cd, (uint32_t)(cd >> 32));
-        }
+        uint2 o[3];
+        chunk_codes3<DT, C0, C1, C2>(v, inv2, o);
+        store_codes<C0>(es.codes[0], (size_t)i, o[0]);
+        if (C1 >= 0) store_codes<(C1 >= 0 ? C1 : 0)>(es.codes[1], (size_t)i, o[1]);
+        if (C2 >= 0) store_codes<(C2 >= 0 ? C2 : 0)>(es.codes[2], (size_t)i, o[2]);
     }
     if (status) atomicOr(&hdr->status, status);
 }
@@ -1112,7 +1137,7 @@ int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st, bool cha
     if (x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
     const long long total = x.rows * (x.cols / 8);
-    const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
+    const int grid = (int)std::max<long long>(1, std::min<long long>((total + 1023) / 1024, (long long)sm_count() * 8));   // four loads in flight per thread
     if (x.dtype == MOFQ_F16)
         MOFQ_CUDA_OK(launch_chained(kq_absmax<0>, dim3(grid), dim3(256), 0, st, chained, xp, (long long)x.rows, (int)(x.cols / 8), (long long)x.ld, hdr));
     else
@@ -1182,64 +1207,122 @@ int launch_score(const ScoreJob &job, cudaStream_t st)
     });
 }
 
+namespace {
+
+int emit_class(int format)
+{
+    switch (format) {
+    case MOFQ_INT4: return CLS_INT4;
+    case MOFQ_INT8: return CLS_INT8;
+    case MOFQ_FP8_E4M3: return CLS_E4M3;
+    case MOFQ_FP8_E5M2: return CLS_E5M2;
+    default: return CLS_E2M1;   // both E2M1 variants: same spacing below the IEEE maximum 3 (their Q differ)
+    }
+}
+
+// The emission kernels are instantiated for the class triples one bit-width allows, classes in ascending order.
+template <typename F>
+int dispatch_classes(int dt, int c0, int c1, int c2, F &&f)
+{
+#define MOFQ_CLS(C0_, C1_, C2_)                                                                                     \
+    if (c0 == C0_ && c1 == C1_ && c2 == C2_)                                                                         \
+        return dt == MOFQ_F16 ? f(std::integral_constant<int, 0>(), std::integral_constant<int, C0_>(), std::integral_constant<int, C1_>(), std::integral_constant<int, C2_>()) \
+                              : f(std::integral_constant<int, 1>(), std::integral_constant<int, C0_>(), std::integral_constant<int, C1_>(), std::integral_constant<int, C2_>());
+    MOFQ_CLS(CLS_INT4, -1, -1) MOFQ_CLS(CLS_E2M1, -1, -1) MOFQ_CLS(CLS_INT4, CLS_E2M1, -1) MOFQ_CLS(CLS_E2M1, CLS_E2M1, -1)
+    MOFQ_CLS(CLS_INT4, CLS_E2M1, CLS_E2M1)
+    MOFQ_CLS(CLS_INT8, -1, -1) MOFQ_CLS(CLS_E4M3, -1, -1) MOFQ_CLS(CLS_E5M2, -1, -1) MOFQ_CLS(CLS_INT8, CLS_E4M3, -1)
+    MOFQ_CLS(CLS_INT8, CLS_E5M2, -1) MOFQ_CLS(CLS_E4M3, CLS_E5M2, -1) MOFQ_CLS(CLS_INT8, CLS_E4M3, CLS_E5M2)
+#undef MOFQ_CLS
+    return MOFQ_ERR_UNSUPPORTED;
+}
+
+// The formats of one emission call sorted by class (stable), their buffers following; cls[] padded with -1.
+struct EmitPlan {
+    EmitSet es;
+    int cls[3];
+    bool has_kernel;   // an instantiation exists for the triple (not for a repeated INT or FP8 class)
+};
+int make_emit_plan(int n, const int *formats, void *const *codes, float *const *scales, EmitPlan *plan)
+{
+    if (n < 1 || n > 3) return MOFQ_ERR_UNSUPPORTED;
+    int order[3] = {0, 1, 2};
+    for (int i = 1; i < n; ++i)
+        for (int k = i; k > 0 && emit_class(formats[order[k]]) < emit_class(formats[order[k - 1]]); --k) std::swap(order[k], order[k - 1]);
+    plan->es = EmitSet{};
+    plan->es.n = n;
+    for (int i = 0; i < 3; ++i) plan->cls[i] = -1;
+    int bits = 0;
+    for (int i = 0; i < n; ++i) {
+        FmtDesc d;
+        if (!describe_format(formats[order[i]], &d)) return MOFQ_ERR_INVALID_ARG;
+        if (bits && d.bits != bits) return MOFQ_ERR_INVALID_ARG;   // one code width per call
+        bits = d.bits;
+        plan->cls[i] = emit_class(formats[order[i]]);
+        plan->es.Q[i] = d.Q;
+        plan->es.codes[i] = static_cast<unsigned char *>(codes[order[i]]);
+        plan->es.scales[i] = scales ? scales[order[i]] : nullptr;
+    }
+    plan->has_kernel = dispatch_classes(MOFQ_F16, plan->cls[0], plan->cls[1], plan->cls[2], [](auto, auto, auto, auto) { return MOFQ_OK; }) == MOFQ_OK;
+    return MOFQ_OK;
+}
+
+}  // namespace
+
 // Per-tensor scale from the abs-max already stored in hdr->absmax_bits (launch_absmax); codes of n formats from one read.
 int launch_emit_codes_uniform(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
                               WsHeader *hdr, cudaStream_t st, uint16_t *x16_out, float *alpha_out, bool chained)
 {
-    if (n < 1 || n > 3 || x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
+    if (x.cols / 8 > 0x7fffffffLL) return MOFQ_ERR_UNSUPPORTED;
     if (x16_out && (x.dtype != MOFQ_BF16 || !alpha_out)) return MOFQ_ERR_INVALID_ARG;
-    EmitSet es{};
-    es.n = n;
-    es.x16 = x16_out;
-    es.alpha = alpha_out;
-    for (int i = 0; i < n; ++i) {
-        FmtDesc d;
-        if (!describe_format(formats[i], &d)) return MOFQ_ERR_INVALID_ARG;
-        es.format[i] = formats[i];
-        es.Q[i] = d.Q;
-        es.codes[i] = static_cast<unsigned char *>(codes[i]);
-        es.scales[i] = scales ? scales[i] : nullptr;
+    EmitPlan plan;
+    if (int rc = make_emit_plan(n, formats, codes, scales, &plan)) return rc;
+    if (!plan.has_kernel) {   // a class twice: one launch per format (the binary16 copy with the first)
+        for (int i = 0; i < n; ++i)
+            if (int rc = launch_emit_codes_uniform(x, 1, formats + i, codes + i, scales ? scales + i : nullptr, hdr, st,
+                                                   i == 0 ? x16_out : nullptr, i == 0 ? alpha_out : nullptr, chained || i > 0))
+                return rc;
+        return MOFQ_OK;
     }
+    plan.es.x16 = x16_out;
+    plan.es.alpha = alpha_out;
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
     const long long total = x.rows * (x.cols / 8);
-    const int grid = (int)std::min<long long>((total + 255) / 256, (long long)sm_count() * 8);
+    const int grid = (int)std::max<long long>(1, std::min<long long>((total + 1023) / 1024, (long long)sm_count() * 8));   // >= 4 chunks per thread
     // a dense tensor is one long row for this kernel (the codes are dense either way): no per-chunk row arithmetic
     const bool flat = x.ld == x.cols && total <= 0x7fffffffLL;
     const long long rows = flat ? 1 : x.rows;
     const int cpr = flat ? (int)total : (int)(x.cols / 8);
-    if (x.dtype == MOFQ_F16)
-        MOFQ_CUDA_OK(launch_chained(kq_emit_codes_uniform<0>, dim3(grid), dim3(256), 0, st, chained, xp, rows, cpr, (long long)x.ld, es, hdr));
-    else
-        MOFQ_CUDA_OK(launch_chained(kq_emit_codes_uniform<1>, dim3(grid), dim3(256), 0, st, chained, xp, rows, cpr, (long long)x.ld, es, hdr));
-    return MOFQ_OK;
+    return dispatch_classes(x.dtype, plan.cls[0], plan.cls[1], plan.cls[2], [&](auto DT, auto C0, auto C1, auto C2) {
+        MOFQ_CUDA_OK(launch_chained(kq_emit_codes_uniform<DT(), C0(), C1(), C2()>, dim3(grid), dim3(256), 0, st, chained, xp, rows, cpr,
+                                    (long long)x.ld, plan.es, hdr));
+        return MOFQ_OK;
+    });
 }
 
 // Per-channel abs-max scales; codes (and scales) of n formats from one read.  formats[i] is a mofq_format.
 int launch_emit_codes_rows(const mofq_tensor &x, int n, const int *formats, void *const *codes, float *const *scales,
                            WsHeader *hdr, cudaStream_t st, bool chained)
 {
-    if (n < 1 || n > 3 || x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
+    if (x.cols > (1 << 20)) return MOFQ_ERR_UNSUPPORTED;
     const size_t smem = (size_t)x.cols * 2;
     if (smem > 200 * 1024) return MOFQ_ERR_UNSUPPORTED;
-    EmitSet es{};
-    es.n = n;
-    for (int i = 0; i < n; ++i) {
-        FmtDesc d;
-        if (!describe_format(formats[i], &d)) return MOFQ_ERR_INVALID_ARG;
-        es.format[i] = formats[i];
-        es.Q[i] = d.Q;
-        es.codes[i] = static_cast<unsigned char *>(codes[i]);
-        es.scales[i] = scales ? scales[i] : nullptr;
+    EmitPlan plan;
+    if (int rc = make_emit_plan(n, formats, codes, scales, &plan)) return rc;
+    if (!plan.has_kernel) {   // a class twice: one launch per format
+        for (int i = 0; i < n; ++i)
+            if (int rc = launch_emit_codes_rows(x, 1, formats + i, codes + i, scales ? scales + i : nullptr, hdr, st, chained || i > 0)) return rc;
+        return MOFQ_OK;
     }
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
-    auto launch = [&](auto kernel) {
+    return dispatch_classes(x.dtype, plan.cls[0], plan.cls[1], plan.cls[2], [&](auto DT, auto C0, auto C1, auto C2) {
+        auto kernel = kq_emit_codes_rows<DT(), C0(), C1(), C2()>;
         if (int rc = set_smem(kernel, smem)) return rc;
         const int occ = std::max(1, blocks_per_sm((const void *)kernel, kRowThreads, smem));
         const int grid = (int)std::min<long long>(x.rows, (long long)sm_count() * occ);
-        MOFQ_CUDA_OK(launch_chained(kernel, dim3(grid), dim3(kRowThreads), smem, st, chained, xp, (long long)x.rows, (int)x.cols, (long long)x.ld, es, hdr));
+        MOFQ_CUDA_OK(launch_chained(kernel, dim3(grid), dim3(kRowThreads), smem, st, chained, xp, (long long)x.rows, (int)x.cols, (long long)x.ld,
+                                    plan.es, hdr));
         return MOFQ_OK;
-    };
-    return x.dtype == MOFQ_F16 ? launch(kq_emit_codes_rows<0>) : launch(kq_emit_codes_rows<1>);
+    });
 }
 
 int launch_emit(const mofq_tensor &x, const FmtDesc &f, int gran, int group, const float *scales_in, void *codes_out,
