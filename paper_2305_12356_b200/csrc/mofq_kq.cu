@@ -1138,10 +1138,14 @@ int launch_absmax(const mofq_tensor &x, WsHeader *hdr, cudaStream_t st, bool cha
     const uint16_t *xp = static_cast<const uint16_t *>(x.data);
     const long long total = x.rows * (x.cols / 8);
     const int grid = (int)std::max<long long>(1, std::min<long long>((total + 1023) / 1024, (long long)sm_count() * 8));   // four loads in flight per thread
+    // a dense tensor is one long row for the kernel: no per-chunk row arithmetic, independent loads
+    const bool flat = x.ld == x.cols && total <= 0x7fffffffLL;
+    const long long rows = flat ? 1 : x.rows;
+    const int cpr = flat ? (int)total : (int)(x.cols / 8);
     if (x.dtype == MOFQ_F16)
-        MOFQ_CUDA_OK(launch_chained(kq_absmax<0>, dim3(grid), dim3(256), 0, st, chained, xp, (long long)x.rows, (int)(x.cols / 8), (long long)x.ld, hdr));
+        MOFQ_CUDA_OK(launch_chained(kq_absmax<0>, dim3(grid), dim3(256), 0, st, chained, xp, rows, cpr, (long long)x.ld, hdr));
     else
-        MOFQ_CUDA_OK(launch_chained(kq_absmax<1>, dim3(grid), dim3(256), 0, st, chained, xp, (long long)x.rows, (int)(x.cols / 8), (long long)x.ld, hdr));
+        MOFQ_CUDA_OK(launch_chained(kq_absmax<1>, dim3(grid), dim3(256), 0, st, chained, xp, rows, cpr, (long long)x.ld, hdr));
     return MOFQ_OK;
 }
 

@@ -583,19 +583,30 @@ struct LayerFinalize {
     uint32_t *absmax_bits;   // the header's activation abs-max: left zero for the next layer of the call
 };
 
-__global__ void __launch_bounds__(32)
+// Warp k adds entry k's partial sums (the reference's, then one per candidate) in a fixed order: lane l takes blocks
+// l, l + 32, ..., eight of them fetched per trip, then the lanes' sums are folded.
+constexpr int kFinalizeThreads = 32 * (1 + MOFQ_MAX_CAND);
+__global__ void __launch_bounds__(kFinalizeThreads)
 layer_finalize(const LayerFinalize f)
 {
     chain_enter();
+    __shared__ double tot[1 + MOFQ_MAX_CAND];
+    const int k = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) *f.absmax_bits = 0;
-    double tot[1 + MOFQ_MAX_CAND];
-    for (int k = 0; k <= f.n_cand; ++k) {
+    if (k <= f.n_cand) {
         double s = 0.0;
-        for (int c = threadIdx.x; c < f.n_ctas[k]; c += 32) s += f.partials[(size_t)k * f.stride + c];
+        for (int c0 = lane; c0 < f.n_ctas[k]; c0 += 32 * 8) {
+            double v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = c0 + 32 * j < f.n_ctas[k] ? __ldcg(&f.partials[(size_t)k * f.stride + c0 + 32 * j]) : 0.0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s += v[j];
+        }
 #pragma unroll
         for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        tot[k] = s;
+        if (lane == 0) tot[k] = s;
     }
+    __syncthreads();
     if (threadIdx.x != 0) return;
     double best = INFINITY, second = INFINITY;
     int chosen = -1;
@@ -975,7 +986,7 @@ int layer_metric_run(const mofq_layer &L, const mofq_config *cfg, mofq_result *r
     f.absmax_bits = &hdr->absmax_bits;
     // (after the per-candidate loop of the general path the previous launch may be a memset-preceded kernel of the
     // emission path: a chained launch behind a kernel that never signals simply starts when that kernel has finished)
-    if (launch_chained(layer_finalize, dim3(1), dim3(32), 0, st, true, f) != cudaSuccess) {
+    if (launch_chained(layer_finalize, dim3(1), dim3(kFinalizeThreads), 0, st, true, f) != cudaSuccess) {
         (void)cudaGetLastError();
         return MOFQ_ERR_CUDA;
     }
