@@ -1224,7 +1224,8 @@ int emit_class(int format)
     }
 }
 
-// The emission kernels are instantiated for the class triples one bit-width allows, classes in ascending order.
+// The emission kernels are instantiated for single classes and for the 8-bit class pairs and triple, classes in
+// ascending order; any other list is emitted one format per launch.
 template <typename F>
 int dispatch_classes(int dt, int c0, int c1, int c2, F &&f)
 {
@@ -1232,8 +1233,7 @@ int dispatch_classes(int dt, int c0, int c1, int c2, F &&f)
     if (c0 == C0_ && c1 == C1_ && c2 == C2_)                                                                         \
         return dt == MOFQ_F16 ? f(std::integral_constant<int, 0>(), std::integral_constant<int, C0_>(), std::integral_constant<int, C1_>(), std::integral_constant<int, C2_>()) \
                               : f(std::integral_constant<int, 1>(), std::integral_constant<int, C0_>(), std::integral_constant<int, C1_>(), std::integral_constant<int, C2_>());
-    MOFQ_CLS(CLS_INT4, -1, -1) MOFQ_CLS(CLS_E2M1, -1, -1) MOFQ_CLS(CLS_INT4, CLS_E2M1, -1) MOFQ_CLS(CLS_E2M1, CLS_E2M1, -1)
-    MOFQ_CLS(CLS_INT4, CLS_E2M1, CLS_E2M1)
+    MOFQ_CLS(CLS_INT4, -1, -1) MOFQ_CLS(CLS_E2M1, -1, -1)   // (4-bit codes are emitted one format at a time: no caller asks for more)
     MOFQ_CLS(CLS_INT8, -1, -1) MOFQ_CLS(CLS_E4M3, -1, -1) MOFQ_CLS(CLS_E5M2, -1, -1) MOFQ_CLS(CLS_INT8, CLS_E4M3, -1)
     MOFQ_CLS(CLS_INT8, CLS_E5M2, -1) MOFQ_CLS(CLS_E4M3, CLS_E5M2, -1) MOFQ_CLS(CLS_INT8, CLS_E4M3, CLS_E5M2)
 #undef MOFQ_CLS
@@ -1244,7 +1244,7 @@ int dispatch_classes(int dt, int c0, int c1, int c2, F &&f)
 struct EmitPlan {
     EmitSet es;
     int cls[3];
-    bool has_kernel;   // an instantiation exists for the triple (not for a repeated INT or FP8 class)
+    bool has_kernel;   // an instantiation exists for the triple
 };
 int make_emit_plan(int n, const int *formats, void *const *codes, float *const *scales, EmitPlan *plan)
 {

@@ -52,6 +52,24 @@ def test_layer_output_error_matches_oracle(orc, dev, T, n_in, n_out, names, w_on
     assert rel_err(nsr.cpu().numpy(), want_nsr).max() < LAYER_RTOL, (nsr, want_nsr)
 
 
+@pytest.mark.parametrize("names", [["FP8_E5M2", "INT8"], ["FP8_E4M3", "FP8_E5M2", "INT8"], ["FP8_E5M2", "FP8_E4M3"], ["FP8_E4M3"],
+                                   ["INT8", "FP8_E4M3", "INT8"], ["FP8_E5M2", "FP8_E5M2"]])
+def test_candidate_order_and_repeats_in_the_8bit_setting(orc, dev, names):
+    """The code-emission kernels take the formats in a fixed class order and exist for distinct classes only: any
+    caller's order, and a list that repeats a format, must still give each candidate its own error."""
+    T, n_in, n_out = 256, 512, 384
+    w, x = _layer(dev, T, n_in, n_out, seed=57, layer=3)
+    cfg = mofq.make_config(8, names, metric="layer_output", is_w_only=False, w_gran="channel", a_gran="tensor")
+    mse, nsr, st = mofq.layer_output_error(x, w, cfg)
+    torch.cuda.synchronize()
+    want_mse, want_nsr = _oracle(orc, w, x, names, False)
+    assert int(st.item()) == 0
+    assert rel_err(mse.cpu().numpy(), want_mse).max() < LAYER_RTOL, (mse, want_mse)
+    assert rel_err(nsr.cpu().numpy(), want_nsr).max() < LAYER_RTOL, (nsr, want_nsr)
+    res = mofq.select_formats([(w, x)], cfg)
+    assert res[0]["chosen"] == int(np.argmin(want_mse)) and res[0]["status"] == 0      # (first minimum: strict '<')
+
+
 @pytest.mark.parametrize("T,n_in,n_out", [(512, 1024, 8192), (256, 22016, 512)])
 def test_dense_outlier_activations_paired_tiles_and_full_depth(orc, dev, T, n_in, n_out):
     """Dense calibration activations with outlier channels (the 65B-shaped workload's recipe) at sizes whose cost
