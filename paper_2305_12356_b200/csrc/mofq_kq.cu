@@ -312,7 +312,11 @@ kq_select_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long 
         const float a = mag16_to_float<DT>(m16);
         kqmath::Sc<NC> sc;
 #pragma unroll
-        for (int j = 0; j < NC; ++j) scale_pair(a, rq.q[j], sc.s[j], sc.inv[j], status);
+        for (int j = 0; j < NC; ++j) {
+            // binary16 abs-max values cannot overflow the reciprocal: the short division-free sequence is exact there
+            if (DT == MOFQ_F16) kqmath::scale_pair_fast(a, rq.q[j], rq.rq[j], sc.s[j], sc.inv[j]);
+            else scale_pair(a, rq.q[j], sc.s[j], sc.inv[j], status);
+        }
         S scorer;
         scorer.begin(sc);
         if (one_pass) {
