@@ -273,6 +273,28 @@ int mofq_select_blocks(const mofq_tensor *x, const int32_t *formats, int n, int 
     if (int rc = check_ws(workspace, workspace_bytes, mofq_tensor_workspace_bytes(x))) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return MOFQ_ERR_CUDA;
+    // a large dense tensor with group-128 blocks: the TMA-fed persistent kernel, as a list of one layer, in its
+    // block-wise form (smaller tensors, other block widths and strided ones: the register-resident kernel below)
+    if (gran == MOFQ_PER_GROUP && mt_blocks_applicable(*x, group, cs, fp_formats) && sizeof(WsHeader) + mt_ws_bytes(1) <= score_ws_bytes()) {
+        mofq_config cfg{};
+        cfg.bit_width = d0.bits;
+        cfg.n_candidates = n;
+        for (int i = 0; i < n; ++i) cfg.candidates[i] = formats[i];
+        cfg.is_w_only = 1;
+        cfg.w_gran = MOFQ_PER_GROUP;
+        cfg.w_gran2 = MOFQ_GRAN_NONE;
+        cfg.w_group = group;
+        cfg.metric = MOFQ_TENSOR_MSE;
+        mofq_layer one{};
+        one.W = *x;
+        BlockSel bs{};
+        bs.choice = choice_out;
+        bs.block_sse = block_sse_out;
+        bs.n_cand = n;
+        std::memcpy(bs.perm, perm, sizeof(bs.perm));
+        return mt_run(&one, 1, &cfg, cs, perm, nc, fp_formats, nullptr, static_cast<char *>(workspace) + sizeof(WsHeader), st, mse_out,
+                      &static_cast<WsHeader *>(workspace)->status, &bs);
+    }
     ScoreJob job{};
     job.x = *x;
     job.cs = cs;

@@ -104,6 +104,14 @@ struct Finalize {
     double inv_n;          // 1 / element count
 };
 
+// Outputs of block-wise selection (one winner per scale block).
+struct BlockSel {
+    uint8_t *choice;     // [blocks] index into the caller's candidate list
+    float *block_sse;    // nullable: [blocks][n_cand], caller's order
+    int n_cand;
+    int perm[MOFQ_MAX_CAND];   // caller's candidate index -> canonical slot
+};
+
 struct ScoreJob {
     mofq_tensor x;
     CandSet cs;
@@ -137,9 +145,13 @@ struct MtLayer {
 // multi-tensor path (mofq_kq_mt.cu)
 bool mt_applicable(const mofq_layer *layers, int n_layers, const mofq_config *cfg);
 size_t mt_ws_bytes(int n_layers);
+// bs (one dense tensor with group-128 scales only): also pick a winner per group; mse_out then has one more entry, the
+// error of the mixture.  mt_blocks_applicable says whether that form exists for the candidate set.
+bool mt_blocks_applicable(const mofq_tensor &W, int group, const CandSet &cs, const int *fp_formats);
 int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
            const int *fp_formats, mofq_result *results /* nullable */, void *ws, cudaStream_t st,
-           float *mse_out = nullptr /* [layer][candidate] */, int32_t *status_out = nullptr /* OR of the layers' status bits */);
+           float *mse_out = nullptr /* [layer][candidate] */, int32_t *status_out = nullptr /* OR of the layers' status bits */,
+           const BlockSel *bs = nullptr);
 int sm_count();
 
 // streamed-rows path (mofq_kq_rows.cu): per-channel scales, alone or with group-128 scales from the same read

@@ -256,13 +256,6 @@ kq_score_rows(const uint16_t *__restrict__ x, long long rows, int cols, long lon
 // block at a time, up to four chunks per lane held in registers: abs-max by shuffles, scales, then every candidate's squared error from the same registers; lane 0
 // of the team applies Algorithm 1's rule (strictly smaller, caller's order) to the block's errors.  Accumulators:
 // [canonical slots][mixture].
-struct BlockSel {
-    uint8_t *choice;     // [blocks] index into the caller's candidate list
-    float *block_sse;    // nullable: [blocks][n_cand], caller's order
-    int n_cand;
-    int perm[MOFQ_MAX_CAND];
-};
-
 template <int DT, int NI, int K0, int K1>
 __global__ void __launch_bounds__(256)
 kq_select_blocks(const uint16_t *__restrict__ x, long long rows, int cols, long long ld, int width, int team, RowQ rq,

@@ -53,6 +53,7 @@ struct MtParams {
     double *partials;    // [slot][kMaxAcc]
     int32_t *status;     // [layer]
     int32_t *timeout;    // one word: set if a bounded wait expired
+    BlockSel bs;         // block-wise form (one tensor): the winner of every group, and the groups' errors
 };
 
 __device__ __forceinline__ int find_layer(const MtLayer *layers, int n, long long tile)
@@ -66,12 +67,15 @@ __device__ __forceinline__ int find_layer(const MtLayer *layers, int n, long lon
     return lo;
 }
 
-template <int DT, int NI, int K0, int K1>
+// BLK: a lane also applies Algorithm 1's rule to its group's errors (strictly smaller, caller's order), writes the
+// winner (and the errors), and one more accumulator sums the winners' errors: the error of the mixed-format tensor.
+template <int DT, int NI, int K0, int K1, bool BLK>
 __global__ void __launch_bounds__(kThreads)
 kq_score_mt(const MtParams p)
 {
     using S = Scorer<DT, NI, K0, K1, true>;
     constexpr int NC = S::NC;
+    constexpr int NA = NC + (BLK ? 1 : 0);
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages];
     __shared__ int err;
@@ -133,25 +137,25 @@ kq_score_mt(const MtParams p)
     const int cpg = p.group >> 3;
     MtLayer L = p.layers[layer];
     long long next_begin = layer + 1 < p.n_layers ? p.layers[layer + 1].tile_begin : p.total_tiles;
-    double dacc[NC];
+    double dacc[NA];
 #pragma unroll
-    for (int j = 0; j < NC; ++j) dacc[j] = 0.0;
+    for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
     int status = 0;
 
     auto flush = [&]() {
         // per-warp partial of the finished layer -> its slot; the finalize kernel adds the slots in order
 #pragma unroll
-        for (int j = 0; j < NC; ++j)
+        for (int j = 0; j < NA; ++j)
 #pragma unroll
             for (int o = 16; o; o >>= 1) dacc[j] += __shfl_xor_sync(0xffffffffu, dacc[j], o);
         if (lane == 0) {
             const long long slot = L.slot_off + (long long)(blockIdx.x - L.first_cta) * kConsumerWarps + warp;
 #pragma unroll
-            for (int j = 0; j < NC; ++j) p.partials[slot * kMaxAcc + j] = dacc[j];
+            for (int j = 0; j < NA; ++j) p.partials[slot * kMaxAcc + j] = dacc[j];
         }
         if (status) atomicOr(&p.status[layer], status);
 #pragma unroll
-        for (int j = 0; j < NC; ++j) dacc[j] = 0.0;
+        for (int j = 0; j < NA; ++j) dacc[j] = 0.0;
         status = 0;
     };
 
@@ -200,7 +204,35 @@ kq_score_mt(const MtParams p)
 #pragma unroll 4
                 for (int j = 0; j < cpg; ++j) scorer.chunk(lds128(a0 ^ (uint32_t)(j << 4)));
             }
-            scorer.end(dacc);
+            if (BLK) {
+                const long long b = g0 + g;   // the tensor is dense: its groups are the blocks, row-major
+                double eg[NC];
+#pragma unroll
+                for (int j = 0; j < NC; ++j) eg[j] = 0.0;
+                scorer.end(eg);
+                float e[NC];
+#pragma unroll
+                for (int j = 0; j < NC; ++j) e[j] = (float)eg[j];
+                float best = INFINITY;
+                int pick = 0;
+                for (int i = 0; i < p.bs.n_cand; ++i) {
+                    float ei = e[0];
+#pragma unroll
+                    for (int j = 1; j < NC; ++j)
+                        if (p.bs.perm[i] == j) ei = e[j];
+                    if (p.bs.block_sse) p.bs.block_sse[b * p.bs.n_cand + i] = ei;
+                    if (ei < best) {                            // strictly smaller: the first candidate keeps a tie
+                        best = ei;
+                        pick = i;
+                    }
+                }
+                p.bs.choice[b] = (uint8_t)pick;
+#pragma unroll
+                for (int j = 0; j < NC; ++j) dacc[j] += (double)e[j];
+                dacc[NC] += (double)best;
+            } else {
+                scorer.end(dacc);
+            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty_bar[s]);
@@ -279,10 +311,10 @@ int fp_kind(int format)
     return -1;
 }
 
-template <int DT, int NI, int K0, int K1>
+template <int DT, int NI, int K0, int K1, bool BLK = false>
 int launch(const MtParams &p, int grid, cudaStream_t st)
 {
-    auto kernel = kq_score_mt<DT, NI, K0, K1>;
+    auto kernel = kq_score_mt<DT, NI, K0, K1, BLK>;
     const size_t smem = (size_t)kStages * kTileBytes + 1024;   // + slack to align the tiles
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
         (void)cudaGetLastError();
@@ -305,6 +337,20 @@ int dispatch(int ni, int k0, int k1, const MtParams &p, int grid, cudaStream_t s
     return MOFQ_ERR_UNSUPPORTED;
 }
 
+// The block-wise form exists for INT4 against FP4-E2M1.  (The 8-bit formats stay with the register-resident kernel and
+// its unscaled errors: this kernel forms a group's error in units of the scale, d = r - x * inv, and inv * scale differs
+// from 1 by up to 2^-23; against an 8-bit grid's |x * inv| <= 127 and |d| <= 0.5 that is a few 1e-5 of one group's
+// sum - invisible in a tensor's mean, too much for a single block's reported error.)
+template <int DT>
+int dispatch_blocks(int ni, int k0, int k1, const MtParams *p, int grid, cudaStream_t st)
+{
+#define MOFQ_MTB(K0_, K1_) \
+    if (ni == 1 && k0 == K0_ && k1 == K1_) return p ? launch<DT, 1, K0_, K1_, true>(*p, grid, st) : MOFQ_OK;
+    MOFQ_MTB(FPK_E2M1, -1)
+#undef MOFQ_MTB
+    return MOFQ_ERR_UNSUPPORTED;
+}
+
 size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 int mt_grid() { return sm_count() * kCtasPerSm; }
 
@@ -320,6 +366,13 @@ bool mt_applicable(const mofq_layer *layers, int n_layers, const mofq_config *cf
     return true;
 }
 
+bool mt_blocks_applicable(const mofq_tensor &W, int group, const CandSet &cs, const int *fp_formats)
+{
+    if (group != 128 || W.ld != W.cols || W.rows * W.cols < (8LL << 20)) return false;   // small tensors: the register kernel, one launch
+    const int k0 = cs.n_fp > 0 ? fp_kind(fp_formats[0]) : -1, k1 = cs.n_fp > 1 ? fp_kind(fp_formats[1]) : -1;
+    return dispatch_blocks<MOFQ_F16>(cs.n_int, k0, k1, nullptr, 0, nullptr) == MOFQ_OK;
+}
+
 size_t mt_ws_bytes(int n_layers)
 {
     const size_t slots = ((size_t)mt_grid() + (size_t)n_layers) * kConsumerWarps;
@@ -328,8 +381,10 @@ size_t mt_ws_bytes(int n_layers)
 }
 
 int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const CandSet &cs, const int *perm, int nc,
-           const int *fp_formats, mofq_result *results, void *ws, cudaStream_t st, float *mse_out, int32_t *status_out)
+           const int *fp_formats, mofq_result *results, void *ws, cudaStream_t st, float *mse_out, int32_t *status_out,
+           const BlockSel *bs)
 {
+    if (bs && (n_layers != 1 || !mt_blocks_applicable(layers[0].W, cfg->w_group, cs, fp_formats))) return MOFQ_ERR_UNSUPPORTED;
     const int grid = mt_grid();
     const int gpt = (kTileBytes / 2) / cfg->w_group;
     std::vector<MtLayer> table((size_t)n_layers);
@@ -383,8 +438,15 @@ int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const
     p.timeout = d_status + n_layers;
     const int k0 = cs.n_fp > 0 ? fp_kind(fp_formats[0]) : -1, k1 = cs.n_fp > 1 ? fp_kind(fp_formats[1]) : -1;
     const int used = (int)std::min<long long>(grid, (tiles + tpc - 1) / tpc);
-    int rc = layers[0].W.dtype == MOFQ_F16 ? dispatch<MOFQ_F16>(cs.n_int, k0, k1, p, used, st)
+    int rc;
+    if (bs) {
+        p.bs = *bs;
+        rc = layers[0].W.dtype == MOFQ_F16 ? dispatch_blocks<MOFQ_F16>(cs.n_int, k0, k1, &p, used, st)
+                                           : dispatch_blocks<MOFQ_BF16>(cs.n_int, k0, k1, &p, used, st);
+    } else {
+        rc = layers[0].W.dtype == MOFQ_F16 ? dispatch<MOFQ_F16>(cs.n_int, k0, k1, p, used, st)
                                            : dispatch<MOFQ_BF16>(cs.n_int, k0, k1, p, used, st);
+    }
     if (rc) return rc;
     Finalize fin{};
     fin.n_cand = cfg->n_candidates;
@@ -393,6 +455,12 @@ int mt_run(const mofq_layer *layers, int n_layers, const mofq_config *cfg, const
     fin.mse_out = mse_out;
     fin.status_out = status_out;
     for (int i = 0; i < MOFQ_MAX_CAND; ++i) fin.perm[i] = perm[i];
+    if (bs) {   // the candidates in the caller's order, then the mixture (accumulator nc)
+        if (fin.n_cand + 1 > MOFQ_MAX_CAND) return MOFQ_ERR_UNSUPPORTED;
+        fin.perm[fin.n_cand] = fin.nc;
+        fin.n_cand += 1;
+        fin.nc += 1;
+    }
     kq_mt_finalize<<<n_layers, 128, 0, st>>>(d_table, d_partials, d_status, d_status + n_layers, fin, results);
     if (cudaGetLastError() != cudaSuccess) return MOFQ_ERR_CUDA;
     return MOFQ_OK;

@@ -70,6 +70,24 @@ def test_block_selection_matches_oracle(orc, dev, names, gran, group, dtype):
         assert len(set(choice.tolist())) > 1                                     # the map does mix formats
 
 
+@pytest.mark.parametrize("names,dtype", [(["INT4", "FP4_E2M1"], torch.float16), (["FP4_E2M1", "INT4"], torch.bfloat16),
+                                         (["FP8_E4M3", "INT8"], torch.float16)])
+def test_large_dense_tensor_takes_the_streamed_route(orc, dev, names, dtype):
+    """8 Mi elements and more with group-128 blocks and the 4-bit pair go through the persistent TMA-fed kernel in its
+    block-wise form (the 8-bit pair stays with the register-resident kernel): several tiles per CTA, a ragged last tile
+    (4099 rows), winners that mix, a zero group and a planted Inf's status."""
+    x = _tensor(dev, 4099, 2048, dtype, 36)
+    x[7, 128:256] = 0
+    want, choice = _check(orc, x, names, "group", 128)
+    assert len(set(choice.tolist())) > 1
+    assert choice[7 * 16 + 1] == 0                                                # the zero group: a tie, first candidate
+    again = mofq.select_blocks(x, names, "group", 128, want_block_sse=True)
+    np.testing.assert_array_equal(again["choice"].cpu().numpy(), choice)         # same launch geometry, same sums
+    x[4098, 2047] = float("inf")
+    got = mofq.select_blocks(x, names, "group", 128)
+    assert int(got["status"].item()) & mofq.binding.STATUS_NONFINITE_INPUT
+
+
 def test_block_selection_odd_row_length_and_strided_view(orc, dev):
     full = _tensor(dev, 37, 1000 + 24, torch.float16, 32)
     view = full[:, 16:1016]                                                      # 1000 columns: 125 chunks per row, ld = 1024
