@@ -18,6 +18,10 @@
  *     in a fixed scratch array inside the library (see there).  All work is enqueued on `stream`
  *     (a cudaStream_t passed as void*; NULL = default stream) and the call returns without
  *     synchronising, unless stated.
+ *   - The device entry points enqueue kernels and memsets only, so a call whose arguments stay valid
+ *     can be captured into a CUDA graph and replayed; make one plain call of the same kind first
+ *     (it sets the kernels' function attributes, which is not a stream operation).  The *_host
+ *     variants copy from host memory and synchronise: they are not for capture.
  *   - Return value: 0 on success, a negative MOFQ_ERR_* for a synchronous argument error.  After
  *     a negative return the call's outputs are not produced.  Pointer, size, alignment, enum,
  *     candidate and workspace errors are found before anything is enqueued; a combination that
