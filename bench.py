@@ -358,6 +358,13 @@ def measure(w, args, barrier, peaks, which, steps, warmup, flusher):
            "l2": "L2 flushed between timed steps (each step timed on its own)" if flush else "inputs larger than L2"}
     if flush is not None:
         rec["ms_per_step_l2_resident"] = time_loop(w.step, steps, warmup, barrier, None)
+        # the same call captured once into a CUDA graph and replayed (what a caller bound by launch latency would do)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            w.step()
+        rec["ms_per_step_graph_replay"] = time_loop(graph.replay, steps, warmup, barrier, flush)
+        rec["ms_per_step_graph_replay_l2_resident"] = time_loop(graph.replay, steps, warmup, barrier, None)
+        del graph
     kernel, dom, launches = kernel_facts(w)
     rec["gpu_launches_per_step"] = launches
     recs = B._parse_results(bytes(w.results.cpu().numpy()), w.n_rec, w.cfg.n_candidates)
