@@ -131,6 +131,20 @@ def static_config(workload, blocks=None):
 
 
 # --------------------------------------------------------------------------------------------------
+def host_cpu():
+    """Logical CPUs of the host and its CPU model string (for the oracle's baseline record)."""
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return {"nproc": os.cpu_count(), "cpu_model": model}
+
+
 def cpu_oracle_sample(workload, budget_s=12.0, max_chunks=64):
     """Time the CPU oracle (as it stands) on chunks of the workload's first layers."""
     from oracle import api as orc
@@ -157,7 +171,7 @@ def cpu_oracle_sample(workload, budget_s=12.0, max_chunks=64):
             done_bytes += w.numel() * 2
             chunks += 1
         scale = t_s / wl["tokens"]
-        return {"value": done_bytes / t_total / 1e9 * scale, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+        return {"value": done_bytes / t_total / 1e9 * scale, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "host": host_cpu(),
                 "sample": f"{chunks} slices of {rows} output rows x {t_s} tokens from the first layers, {t_total:.1f} s of CPU "
                           f"work, layer-output criterion; value extrapolated to {wl['tokens']} tokens (x{scale:.4f})"}, done_bytes * scale, t_total
     while t_total < budget_s and chunks < max_chunks:
@@ -171,7 +185,7 @@ def cpu_oracle_sample(workload, budget_s=12.0, max_chunks=64):
         t_total += time.perf_counter() - t0
         done_bytes += w.numel() * 2
         chunks += 1
-    return {"value": done_bytes / t_total / 1e9, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+    return {"value": done_bytes / t_total / 1e9, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "host": host_cpu(),
             "sample": f"{chunks} chunks of <=1024 rows from the first layers ({done_bytes / 1e6:.0f} MB fp16), "
                       f"{t_total:.1f} s of CPU work, tensor-MSE criterion, {len(grans)} scale granularit{'ies' if len(grans) > 1 else 'y'}"}, done_bytes, t_total
 
