@@ -38,8 +38,8 @@ WORKLOAD_ORDER = ["single_4096_w4_channel", "llama7b_w4_group128", "llama13b_w8a
 # DRAM bytes per element of the scoring kernels, from the ncu captures summarised in profiles/ (read + write bytes
 # over the elements of the captured case; traffic is proportional to the elements processed).  None: not captured
 # for the kernel as it stands.
-DRAM_BYTES_PER_ELEMENT = {"kq_score_mt": (809.57e6 + 4.63e6) / 404750336,          # 14 layers of the 7B-shaped model
-                          "kq_score_rows_mt": (2140.23e6 + 4.79e6) / 1070071808}  # 14 layers of the 33B-shaped model
+DRAM_BYTES_PER_ELEMENT = {"kq_score_mt": (809.61e6 + 3.57e6) / 404750336,          # 14 layers of the 7B-shaped model
+                          "kq_score_rows_mt": (2140.22e6 + 4.90e6) / 1070071808}  # 14 layers of the 33B-shaped model
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 L2_BYTES = 126e6
