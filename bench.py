@@ -588,7 +588,7 @@ def main():
                                              "note": "median of 5 steps launched alone after 50 ms idle (no power-cap throttling); context only"}
 
     if rank == 0 and w.grans == ("group",) and not w.layer_metric and not w.streaming and w.fp16_bytes < 40e9:
-        head["emit_winners_ms"] = emit_winners_ms(w, barrier)
+        head["emit_winners_ms"] = emit_winners_ms(w, torch.cuda.synchronize)   # rank 0 alone: no collective in its barrier
     e2e = None
     if not args.no_e2e:
         e2e = e2e_pass(w, args, dev, barrier, world)
