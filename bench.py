@@ -355,10 +355,10 @@ def kernel_facts(w):
         # per layer besides the products: activation abs-max, weight codes, activation codes (+ fp16 copy), finalize
         return "gemm_err_kernel", n * gemm, n * (gemm + 4) + (2 * n if w.streaming else 0)
     if w.grans == ("group",):
-        return "kq_score_mt", 1, 2 + (n + 63) // 64        # table uploads (64 layers each) + persistent kernel + finalize
+        return "kq_score_mt", 1, 2 + (n + 511) // 512      # table uploads (512 layers each) + persistent kernel + finalize
     if n == 1:
         return "kq_score_rows_mt", 1, 2                    # header clear + scoring launch (its last block applies Algorithm 1's comparison)
-    return "kq_score_rows_mt", 1, 2 + (n + 31) // 32
+    return "kq_score_rows_mt", 1, 2 + (n + 255) // 256     # table uploads (256 layers each) + persistent kernel + finalize
 
 
 def measure(w, args, barrier, peaks, which, steps, warmup, flusher):

@@ -289,9 +289,10 @@ kq_mt_finalize(const MtLayer *layers, const double *partials, int32_t *status, c
     if (fin.status_out && r.status) atomicOr(fin.status_out, r.status);
 }
 
-// The work table travels to the device as kernel arguments, 64 entries per launch: fully stream-ordered,
+// The work table travels to the device as kernel arguments, 512 entries per launch: fully stream-ordered,
 // no pageable-memory copy (which would synchronise the stream) and nothing for the caller to keep alive.
-constexpr int kUploadChunk = 64;
+constexpr int kUploadChunk = 512;   // 24 KB of the 32 KB a launch's parameters may take
+static_assert(sizeof(MtLayer) * kUploadChunk + 64 <= 32764, "the chunk must fit a launch's parameter space");
 struct TableChunk {
     MtLayer e[kUploadChunk];
 };

@@ -480,9 +480,11 @@ kq_rows_finalize(const RmLayer *layers, const double *partials, const int32_t *s
     }
 }
 
-// The work table travels to the device as kernel arguments, a few entries per launch: fully stream-ordered,
-// no pageable-memory copy (which would synchronise the stream) and nothing for the caller to keep alive.
-constexpr int kRmUploadChunk = 32;
+// The work table travels to the device as kernel arguments, 256 entries (26 KB of the 32 KB a launch may carry) per
+// launch: fully stream-ordered, no pageable-memory copy (which would synchronise the stream) and nothing for the caller
+// to keep alive.
+constexpr int kRmUploadChunk = 256;
+static_assert(sizeof(RmLayer) * kRmUploadChunk + 64 <= 32764, "the chunk must fit a launch's parameter space");
 struct RmTableChunk {
     RmLayer e[kRmUploadChunk];
 };
