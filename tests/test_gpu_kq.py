@@ -446,6 +446,26 @@ def test_streamed_rows_random_layer_lists(orc, dev, seed):
                     assert r["chosen"] == orc.select(want), (shapes[i], g, r, want)
 
 
+@pytest.mark.parametrize("g1,g2,n_layers", [("channel", "group", 601), ("group", None, 1100)])
+def test_layer_lists_longer_than_one_table_upload(orc, dev, g1, g2, n_layers):
+    """The work table reaches the device as kernel parameters, a few hundred entries per launch: lists that need
+    three launches (the last one partly filled) must give every layer what that layer gives alone."""
+    names = ["INT4", "FP4_E2M1"]
+    base = [_weights(dev, r, c, seed=66, layer=i) for i, (r, c) in enumerate([(3, 256), (1, 128), (5, 384), (2, 1024), (7, 128)])]
+    xs = [base[i % len(base)] for i in range(n_layers)]
+    cfg = mofq.make_config(4, names, w_gran=g1, w_group=128, w_gran2=g2)
+    recs = mofq.select_formats(xs, cfg)
+    n_sets = 2 if g2 else 1
+    assert len(recs) == n_layers * n_sets
+    for s, g in enumerate((g1, g2)[:n_sets]):
+        for k, x in enumerate(base):
+            want = _oracle_mse(orc, host(x), names, g, 128 if g == "group" else 0)
+            for i in range(k, n_layers, len(base)):
+                r = recs[i * n_sets + s]
+                assert r["status"] == 0 and rel_err(r["errors"], want).max() < MSE_RTOL, (i, g, r, want)
+            assert all(recs[i * n_sets + s] == recs[k * n_sets + s] for i in range(k, n_layers, len(base)))
+
+
 def test_streamed_rows_layers_of_one_call_overlap_safely(orc, dev):
     """Within one selection call the streamed-row kernel lets the next layer's launch start before the current one has
     drained; the header and the partial sums they share are only touched after the earlier launch has completed.
