@@ -604,8 +604,7 @@ def main():
                 continue
             ow = Workload(name, dev, 0)
             steps = max(1, min(args.steps, 3 if ow.streaming else 10 if ow.layer_metric else 50))
-            # (short steps get more warm-up calls: after the previous workload's teardown the clocks need tens of ms to settle)
-            rec = measure(ow, args, barrier, peaks, which, steps, 3 if ow.layer_metric else 20, flusher)
+            rec = measure(ow, args, barrier, peaks, which, steps, 3, flusher)
             rec["config_index"] = WORKLOAD_ORDER.index(name) + 1
             if ow.grans == ("group",) and not ow.layer_metric:
                 rec["emit_winners_ms"] = emit_winners_ms(ow, barrier)
